@@ -1,0 +1,9 @@
+"""fp64 CPU oracle for the CritiPrefill prefill hot path.
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by __graft_entry__.smoke() and by
+bench.py's CPU-baseline legs.  The CUDA product path never imports it, and it
+imports nothing from the CUDA package.
+"""
+from .estimation import summaries, logits, estimate, causal_block_mask  # noqa: F401
+from .selection import select  # noqa: F401
+from .attention import sparse_attention, dense_attention, sparse_attention_rows, dense_attention_rows  # noqa: F401

@@ -1,0 +1,111 @@
+"""Oracle: segment-wise criticality estimation (Algorithm 1), fp64, plain numpy.
+
+TEST INFRASTRUCTURE -- a slow, literal restatement of Algorithm 1 used to check the CUDA
+kernels.  Not part of the product path.
+
+Pins (tests/test_oracle_estimation.py): bit-exact summaries against an explicit token
+loop; row sums of the four softmax maps; agreement of the log-domain result with the
+probability-domain formulas of Algorithm 1 (lines 9-14) evaluated in long double on
+small inputs; the segment = block = 1 special case (a plain library softmax of q K^T,
+i.e. Eq. 3 without the top-k); alpha = 1 and S' = S identities of the fusion step;
+brute-force mask.
+
+Readings of the paper taken here (the paper prints no worked example, so the choice
+among them is "parity unpinned" with respect to the authors' implementation):
+  * scores are kept as natural logarithms ln S in fp64 (the probabilities of Algorithm 1
+    underflow at 128K tokens; ordering and the fusion are unchanged);
+  * the estimation logits carry no 1/sqrt(d) unless est_scale says so (Algorithm 1,
+    lines 9-10, as written);
+  * softmax over all n2 blocks first, causal mask afterwards (lines 9-13 in order);
+    ``mask_before_softmax`` gives the other order;
+  * a block is masked iff it starts at or after the end of the segment;
+  * every query head has its own score map, using the key summaries of its KV group;
+  * S' = None means no fusion; the fused S is what the next layer receives.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+LN2 = float(np.log(2.0))
+
+
+def _f64(x) -> np.ndarray:
+    if hasattr(x, "detach"):
+        x = x.detach().cpu()
+        x = x.float().numpy() if x.dtype.is_floating_point and x.element_size() < 4 else x.numpy()
+    return np.asarray(x, dtype=np.float64)
+
+
+def summaries(Q, K, segment_size: int, block_size: int):
+    """Algorithm 1, lines 3-8: element-wise max / min over the tokens of each query
+    segment and of each key block.  Q [B,Hq,n,d], K [B,Hkv,n,d] ->
+    Qmax,Qmin [B,Hq,n1,d]; Kmax,Kmin [B,Hkv,n2,d]."""
+    Q = _f64(Q)
+    K = _f64(K)
+    B, Hq, n, d = Q.shape
+    Hkv = K.shape[1]
+    assert n % segment_size == 0 and n % block_size == 0
+    n1, n2 = n // segment_size, n // block_size
+    Qr = Q.reshape(B, Hq, n1, segment_size, d)
+    Kr = K.reshape(B, Hkv, n2, block_size, d)
+    return Qr.max(axis=3), Qr.min(axis=3), Kr.max(axis=3), Kr.min(axis=3)
+
+
+def logits(Qrep: np.ndarray, Krep: np.ndarray, est_scale: float = 1.0) -> np.ndarray:
+    """Algorithm 1, lines 9-10 (argument of the softmax): whole-vector dot products of a
+    query representative with every key representative of its KV group.
+    Qrep [B,Hq,n1,d], Krep [B,Hkv,n2,d] -> [B,Hq,n1,n2]."""
+    B, Hq, n1, d = Qrep.shape
+    Hkv = Krep.shape[1]
+    g = Hq // Hkv
+    out = np.empty((B, Hq, n1, Krep.shape[2]), dtype=np.float64)
+    for b in range(B):
+        for h in range(Hq):
+            out[b, h] = est_scale * (Qrep[b, h] @ Krep[b, h // g].T)
+    return out
+
+
+def _logsumexp(x: np.ndarray, axis: int = -1) -> np.ndarray:
+    m = np.max(x, axis=axis, keepdims=True)
+    m = np.where(np.isfinite(m), m, 0.0)
+    with np.errstate(divide="ignore"):
+        return m + np.log(np.sum(np.exp(x - m), axis=axis, keepdims=True))
+
+
+def _logaddexp(a: np.ndarray, b: np.ndarray) -> np.ndarray:
+    with np.errstate(invalid="ignore"):
+        return np.logaddexp(a, b)  # (-inf, -inf) -> -inf
+
+
+def causal_block_mask(n1: int, n2: int, segment_size: int, block_size: int) -> np.ndarray:
+    """True where block b lies entirely in the future of segment j (Algorithm 1, line 13):
+    its first token b*blk is not before the segment's end (j+1)*seg."""
+    j = np.arange(n1)[:, None]
+    b = np.arange(n2)[None, :]
+    return b * block_size >= (j + 1) * segment_size
+
+
+def estimate(Q, K, segment_size: int, block_size: int, *, est_scale: float = 1.0,
+             alpha: float = 0.25, S_prev: np.ndarray | None = None,
+             mask_before_softmax: bool = False) -> np.ndarray:
+    """Algorithm 1 in full.  Returns ln S, shape [B,Hq,n1,n2], fp64; masked entries -inf.
+
+    ``S_prev`` is the ln S returned for the previous layer (None: first layer, no fusion).
+    """
+    Qmax, Qmin, Kmax, Kmin = summaries(Q, K, segment_size, block_size)          # lines 3-8
+    n1, n2 = Qmax.shape[2], Kmax.shape[2]
+    masked = causal_block_mask(n1, n2, segment_size, block_size)
+    L = []
+    for qrep, krep in ((Qmax, Kmax), (Qmax, Kmin), (Qmin, Kmax), (Qmin, Kmin)):   # S1..S4, lines 9-10
+        l = logits(qrep, krep, est_scale)
+        if mask_before_softmax:
+            l = np.where(masked, -np.inf, l)
+        L.append(l - _logsumexp(l, axis=-1))                                     # ln softmax over blocks
+    Lmax = _logaddexp(L[0], L[2]) - LN2                                          # line 11: (S1+S3)/2
+    Lmin = _logaddexp(L[1], L[3]) - LN2                                          #          (S2+S4)/2
+    Lg = np.maximum(Lmax, Lmin)                                                  # line 12
+    Lg = np.where(masked, -np.inf, Lg)                                           # line 13
+    if S_prev is not None and alpha != 1.0:                                      # line 14
+        Lprev = np.asarray(S_prev, dtype=np.float64)
+        Lg = _logaddexp(np.log(alpha) + Lg, np.log1p(-alpha) + Lprev)            # ln(a*S + (1-a)*S')
+    return Lg
