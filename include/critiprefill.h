@@ -1,0 +1,136 @@
+/* critiprefill.h -- C ABI of the B200 (sm_100a) CritiPrefill prefill hot path.
+ *
+ * The library computes, for one attention layer,
+ *   (1) segment-wise query criticality  ln S[j,b]   (paper Algorithm 1),
+ *   (2) the per-segment critical block list          (Algorithm 2, line 8),
+ *   (3) causal GQA attention over the listed blocks  (Algorithm 2, lines 6-13),
+ * and, as the baseline the method is compared with, dense causal attention (Eq. 2).
+ *
+ * General conventions
+ *   - Every pointer argument except `p`, `bytes_out` and `status_out` is a DEVICE pointer
+ *     owned by the caller.  The library allocates no device memory, frees nothing and keeps
+ *     no state between calls.
+ *   - Calls validate their arguments on the host, enqueue kernels on `cuda_stream`
+ *     (a cudaStream_t passed as void*; NULL = the default stream) and return without
+ *     synchronising.  Outputs are valid once the stream reaches that point.
+ *   - Return value: a cp_status.  Conditions only the device can see (a block list that
+ *     breaks its contract, a pipeline wait that ran out) are recorded in the first word of
+ *     the workspace; read it with critiprefill_device_status.  Kernels never trap or assert.
+ *   - Tensor layout: Q and O are [batch, n_q_heads, seq_len, head_dim], K and V are
+ *     [batch, n_kv_heads, seq_len, head_dim]; the three outer strides are given in ELEMENTS
+ *     in cp_params, head_dim is contiguous.  Base pointers must be 16-byte aligned and the
+ *     strides multiples of 8 elements (bf16) / 4 elements (fp32).
+ *   - Notation: n1 = seq_len / segment_size, n2 = seq_len / block_size,
+ *     r = segment_size / block_size (blocks that overlap a segment), k = budget_blocks,
+ *     g = n_q_heads / n_kv_heads; query head h uses KV head h / g.
+ *   - Requirements (else CP_ERR_SHAPE): seq_len % segment_size == 0,
+ *     segment_size % block_size == 0, n_q_heads % n_kv_heads == 0, r <= k <= n2.
+ *   - Supported (else CP_ERR_UNSUPPORTED): head_dim 64 or 128; n2 <= 4096 for estimate;
+ *     the tensor-core attention path needs bf16, head_dim 128, segment_size % 256 == 0 and
+ *     block_size in {32, 64, 128}; everything else runs on a plain SIMT kernel.
+ */
+#ifndef CRITIPREFILL_H_
+#define CRITIPREFILL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CP_OK = 0,
+  CP_ERR_NULL = 1,        /* a required pointer is NULL */
+  CP_ERR_SHAPE = 2,       /* sizes violate the divisibility / range requirements */
+  CP_ERR_UNSUPPORTED = 3, /* valid problem outside the implemented envelope */
+  CP_ERR_WORKSPACE = 4,   /* ws is NULL, misaligned (256 B) or smaller than workspace_bytes */
+  CP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
+  CP_ERR_TIMEOUT = 6,     /* device: a bounded pipeline wait expired; outputs are invalid */
+  CP_ERR_BOUNDS = 7       /* device: a block list broke its contract; that segment was skipped */
+} cp_status;
+
+typedef enum { CP_BF16 = 0, CP_F32 = 1 } cp_dtype;
+
+enum {
+  CP_FLAG_MASK_BEFORE_SOFTMAX = 1, /* estimate: normalise each score map over visible blocks only */
+  CP_FLAG_FORCE_SIMT = 2           /* attention: use the SIMT kernel even where tensor cores apply */
+};
+
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, seq_len, head_dim;
+  int32_t segment_size, block_size, budget_blocks; /* k = budget tokens / block_size */
+  int32_t dtype;                                   /* cp_dtype of Q, K, V, O */
+  int32_t flags;                                   /* CP_FLAG_* */
+  int64_t q_stride[3], k_stride[3], v_stride[3], o_stride[3]; /* batch, head, token (elements) */
+  float est_scale; /* multiplies the four estimation logits; 1.0 = Algorithm 1 as printed */
+  float sm_scale;  /* attention logit scale, 1/sqrt(head_dim) in Eq. 2 / Algorithm 2 line 10 */
+  float alpha;     /* layer-fusion weight of the current layer (Algorithm 1 line 14; 0.25 in
+                      Section 3.1.3); ignored when S_prev is NULL */
+  int32_t reserved;
+} cp_params;
+
+/* Bytes of scratch (`ws`) the calls below need for these parameters; the same buffer serves
+ * all of them.  `ws` must be 256-byte aligned.  Its first 256 bytes are the device status
+ * block, which the caller zeroes once (cudaMemset) before the first call.  Host pointers. */
+int critiprefill_workspace_bytes(const cp_params* p, size_t* bytes_out);
+
+/* Algorithm 1 (estimation of query criticality in one layer).
+ *   Q, K    in   device, layout above.  V is not read by Algorithm 1.
+ *   S_prev  in   device, nullable: ln S returned for the previous layer, [B,Hq,n1,n2] fp64.
+ *                NULL = first layer / no fusion (alpha treated as 1).
+ *   S_out   out  device, [B,Hq,n1,n2] fp64: NATURAL LOG of the criticality score,
+ *                ln( alpha*S + (1-alpha)*S' ); blocks that start at or after the end of the
+ *                segment (causal mask, line 13) hold -inf.  May not alias S_prev.
+ * Steps: per-channel max/min of each query segment and key block (lines 3-8) into ws, four
+ * dot-product logit maps scaled by est_scale and their row softmaxes over all n2 blocks
+ * (lines 9-10), (S1+S3)/2, (S2+S4)/2 and their maximum (lines 11-12), mask (13), fusion (14).
+ * Arithmetic: fp64 on the representatives (which are exact in the input dtype). */
+int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, const double* S_prev,
+                          double* S_out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Algorithm 2, line 8: I_j = argtop_k(S[j], k) with the diagonal blocks always kept.
+ *   S    in   device, [B,Hq,n1,n2] fp64 (as written by critiprefill_estimate)
+ *   idx  out  device, [B,Hq,n1,k] int32: ascending block indices; the r blocks overlapping
+ *             segment j ([j*r,(j+1)*r)) are always present and count against k; the other
+ *             k-r entries are the strictly-past blocks with the largest S[j,b], ties to the
+ *             larger b; entries beyond cnt are -1
+ *   cnt  out  device, [B,Hq,n1] int32 = min(k, (j+1)*r)
+ * Exact (comparisons only). */
+int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws,
+                        size_t ws_bytes, void* cuda_stream);
+
+/* Algorithm 2, lines 6-13, with token-level causality inside the listed blocks:
+ *   O[t] = sum_{u in U_t} softmax_u(sm_scale * q_t.k_u) v_u,
+ *   U_t  = { u <= t : floor(u/block_size) in idx[b,h,j,0:cnt] },  j = floor(t/segment_size).
+ *   Q, K, V   in   device
+ *   idx, cnt  in   device, as produced by critiprefill_select.  Contract per list: ascending,
+ *                  unique, r <= cnt <= k, and its last r entries are exactly the diagonal
+ *                  blocks j*r .. (j+1)*r-1.  A list that breaks it sets CP_ERR_BOUNDS in the
+ *                  status block and its segment's rows of O are not written.
+ *   O         out  device, same dtype and layout family as Q (o_stride)
+ *   lse       out  device, nullable, [B,Hq,n] fp32: ln sum_{u in U_t} exp(sm_scale*q_t.k_u)
+ * bf16: operands bf16, fp32 accumulation, probabilities rounded to bf16 before the PV
+ * product, O rounded to bf16.  fp32: plain fp32 arithmetic. */
+int critiprefill_attention(const cp_params* p, const void* Q, const void* K, const void* V,
+                           const int32_t* idx, const int32_t* cnt, void* O, float* lse, void* ws,
+                           size_t ws_bytes, void* cuda_stream);
+
+/* Eq. 2 with the causal mask (U_t = { u <= t }): the dense baseline, built on the same
+ * pipeline as critiprefill_attention.  Arguments as above; segment_size / block_size /
+ * budget_blocks are ignored apart from the shape requirements. */
+int critiprefill_dense_attention(const cp_params* p, const void* Q, const void* K, const void* V,
+                                 void* O, float* lse, void* ws, size_t ws_bytes,
+                                 void* cuda_stream);
+
+/* Synchronises `cuda_stream`, copies the device status word (a cp_status: CP_OK, CP_ERR_TIMEOUT
+ * or CP_ERR_BOUNDS; sticky until the caller zeroes the status block) to *status_out (host). */
+int critiprefill_device_status(const void* ws, int32_t* status_out, void* cuda_stream);
+
+/* Static, NUL-terminated description of a cp_status value. */
+const char* critiprefill_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CRITIPREFILL_H_ */

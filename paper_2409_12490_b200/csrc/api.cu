@@ -1,0 +1,123 @@
+// The C ABI (include/critiprefill.h): argument validation and kernel dispatch.
+#include "cp_common.cuh"
+
+namespace {
+
+using namespace cp;
+
+int validate(const cp_params* p, Dims* out) {
+  if (p == nullptr) return CP_ERR_NULL;
+  if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->seq_len <= 0 || p->head_dim <= 0 ||
+      p->segment_size <= 0 || p->block_size <= 0 || p->budget_blocks <= 0)
+    return CP_ERR_SHAPE;
+  if (p->dtype != CP_BF16 && p->dtype != CP_F32) return CP_ERR_UNSUPPORTED;
+  if (p->n_q_heads % p->n_kv_heads) return CP_ERR_SHAPE;
+  if (p->seq_len % p->segment_size || p->segment_size % p->block_size) return CP_ERR_SHAPE;
+  Dims m = make_dims(*p);
+  if (m.k < m.r || m.k > m.n2) return CP_ERR_SHAPE;
+  if (m.d != 64 && m.d != 128) return CP_ERR_UNSUPPORTED;
+  const int64_t align = 16 / m.es;
+  const int64_t* strides[4] = {p->q_stride, p->k_stride, p->v_stride, p->o_stride};
+  for (auto s : strides)
+    for (int i = 0; i < 3; ++i)
+      if (s[i] < 0 || s[i] % align) return CP_ERR_SHAPE;
+  for (auto s : strides)
+    if (s[2] < m.d) return CP_ERR_SHAPE;
+  *out = m;
+  return CP_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_ws(const Dims& m, const void* ws, size_t ws_bytes) {
+  if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 255u) || ws_bytes < ws_layout(m).total)
+    return CP_ERR_WORKSPACE;
+  return CP_OK;
+}
+
+int attention_common(const cp_params* p, const void* Q, const void* K, const void* V, const int32_t* idx,
+                     const int32_t* cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* stream, bool dense) {
+  Dims m;
+  int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  if (!Q || !K || !V || !O || (!dense && (!idx || !cnt))) return CP_ERR_NULL;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O)) return CP_ERR_SHAPE;
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  DeviceStatus* st = static_cast<DeviceStatus*>(ws);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (sm100_path_applies(*p, m)) return launch_attention_sm100(*p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
+  return launch_attention_simt(*p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
+}
+
+}  // namespace
+
+extern "C" {
+
+int critiprefill_workspace_bytes(const cp_params* p, size_t* bytes_out) {
+  if (bytes_out == nullptr) return CP_ERR_NULL;
+  Dims m;
+  const int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  *bytes_out = ws_layout(m).total;
+  return CP_OK;
+}
+
+int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, const double* S_prev, double* S_out,
+                          void* ws, size_t ws_bytes, void* cuda_stream) {
+  Dims m;
+  int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  if (!Q || !K || !S_out) return CP_ERR_NULL;
+  if (!aligned16(Q) || !aligned16(K) || S_out == S_prev) return CP_ERR_SHAPE;
+  if (m.n2 > kMaxBlocksN2) return CP_ERR_UNSUPPORTED;
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if ((rc = launch_summarize(*p, m, Q, K, static_cast<char*>(ws), s)) != CP_OK) return rc;
+  return launch_score(*p, m, static_cast<const char*>(ws), S_prev, S_out, s);
+}
+
+int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws, size_t ws_bytes,
+                        void* cuda_stream) {
+  Dims m;
+  int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  if (!S || !idx || !cnt) return CP_ERR_NULL;
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  return launch_select(*p, m, S, idx, cnt, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int critiprefill_attention(const cp_params* p, const void* Q, const void* K, const void* V, const int32_t* idx,
+                           const int32_t* cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return attention_common(p, Q, K, V, idx, cnt, O, lse, ws, ws_bytes, cuda_stream, false);
+}
+
+int critiprefill_dense_attention(const cp_params* p, const void* Q, const void* K, const void* V, void* O,
+                                 float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+  return attention_common(p, Q, K, V, nullptr, nullptr, O, lse, ws, ws_bytes, cuda_stream, true);
+}
+
+int critiprefill_device_status(const void* ws, int32_t* status_out, void* cuda_stream) {
+  if (ws == nullptr || status_out == nullptr) return CP_ERR_NULL;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int32_t code = 0;
+  if (cudaMemcpyAsync(&code, ws, sizeof(code), cudaMemcpyDeviceToHost, s) != cudaSuccess) return CP_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return CP_ERR_CUDA;
+  *status_out = code;
+  return CP_OK;
+}
+
+const char* critiprefill_status_string(int status) {
+  switch (status) {
+    case CP_OK: return "ok";
+    case CP_ERR_NULL: return "a required pointer is NULL";
+    case CP_ERR_SHAPE: return "sizes, strides or alignment violate the requirements";
+    case CP_ERR_UNSUPPORTED: return "problem outside the implemented envelope";
+    case CP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case CP_ERR_CUDA: return "a CUDA call failed";
+    case CP_ERR_TIMEOUT: return "device: a bounded pipeline wait expired";
+    case CP_ERR_BOUNDS: return "device: a block list broke its contract";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

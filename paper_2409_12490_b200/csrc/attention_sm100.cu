@@ -1,0 +1,576 @@
+// K4 / K5: block-sparse (Algorithm 2, lines 6-13) and dense causal (Eq. 2) attention on the
+// sm_100a tensor cores.  bf16 operands, fp32 accumulation in tensor memory, online softmax.
+//
+// One CTA works on 256 consecutive query rows of one (batch, query head): two 128-row tiles
+// "A" and "B" that share every K/V tile the producer brings in.  Roles (320 threads):
+//   warps 0-3  softmax for tile A (one thread per query row)
+//   warps 4-7  softmax for tile B
+//   warp  8    TMA producer: K/V tiles through a 5-slot ring of 32 KB buffers; a gathered
+//              tile is assembled from 128/blk boxes addressed by the block list
+//   warp  9    MMA issuer: S = Q K^T (operands in shared memory), O += P V (P read from
+//              tensor memory, where the softmax warps overwrite S with bf16 probabilities)
+// Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each.
+// The tile sequence of a unit is: gathered past tiles, contiguous unmasked tiles, then the
+// two diagonal tiles; tile A stops one tile earlier than B.  Every wait is bounded: on
+// expiry the waiter raises a CTA-wide abort flag and CP_ERR_TIMEOUT, and all roles drain.
+#include <cuda.h>
+#include <math_constants.h>
+
+#include "cp_common.cuh"
+
+namespace cp {
+namespace {
+
+constexpr int kD = 128;
+constexpr int kTile = 128;
+constexpr int kHalfBytes = kTile * 64 * 2;   // [128 rows x 64 cols] bf16, 128-byte swizzled
+constexpr int kTileBytes = 2 * kHalfBytes;   // both halves of head_dim
+constexpr int kSlots = 5;
+constexpr int kThreads = 320;
+constexpr int kSmemQ = 0;
+constexpr int kSmemKV = 2 * kTileBytes;
+constexpr int kSmemBar = kSmemKV + kSlots * kTileBytes;
+constexpr int kSmemTotal = kSmemBar + 256 + 1024;   // + alignment slack
+constexpr float kRescaleThreshold = 8.0f;           // in log2 units
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct Bars {
+  unsigned long long q_full;
+  unsigned long long kv_full[kSlots];
+  unsigned long long kv_empty[kSlots];
+  unsigned long long s_full[2];
+  unsigned long long p_full[2];
+  unsigned long long o_done[2];
+  uint32_t tmem_base;
+  volatile int abort_flag;
+};
+
+struct Args {
+  const int32_t* idx;
+  const int32_t* cnt;
+  __nv_bfloat16* O;
+  float* lse;
+  DeviceStatus* st;
+  int B, Hq, Hkv, g, n, seg, blk, k, r, n1;
+  int64_t osb, osh, ost;
+  float sm_scale;
+  int dense;
+};
+
+// ---------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this waiter or another gave up).
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, Bars* bars, DeviceStatus* st,
+                                          int site) {
+  if (mbar_test(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if ((it & 63u) == 0) {
+      if (bars->abort_flag) return false;
+      if (globaltimer() - t0 > kWaitLimitNs) {
+        bars->abort_flag = 1;
+        report(st, CP_ERR_TIMEOUT, site, blockIdx.x, threadIdx.x, int(parity));
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, unsigned long long* bar, int c0,
+                                            int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+      ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+        "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+        "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+        "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]),
+        "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Shared-memory matrix descriptors for 128-byte-swizzled tiles whose rows are 128 bytes
+// (64 bf16) and whose 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_base(uint32_t lbo_bytes) {
+  return (uint64_t(lbo_bytes >> 4) << 16) | (uint64_t(1024 >> 4) << 32) | (uint64_t(1) << 46) | (uint64_t(2) << 61);
+}
+__device__ __forceinline__ uint64_t desc_at(uint64_t base, uint32_t smem_addr) {
+  return base | uint64_t((smem_addr & 0x3FFFFu) >> 4);
+}
+
+// instruction descriptors: D fp32, A/B bf16, M = 128, N = 128; B is K-major for Q K^T and
+// MN-major (head_dim contiguous) for P V
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+
+// ---------------------------------------------------------------- unit geometry
+struct Unit {
+  int b, h, kvh;
+  int q_tok;        // first query row of tile A
+  int n_past;       // listed blocks strictly before the segment
+  int n_past_tiles; // gathered tiles
+  int last_cols;    // valid key columns of the last gathered tile
+  int c_tok, n_cont;// contiguous unmasked tiles: first token, count
+  int d_tok;        // first token of diagonal tile d0 (d1 follows)
+  int T;            // tiles for B; A takes T-1
+  const int32_t* list;
+  int seg_j;
+  bool ok;
+};
+
+__device__ __forceinline__ Unit decode_unit(const Args& a) {
+  Unit u;
+  u.ok = true;
+  u.list = nullptr;
+  long long x = blockIdx.x;
+  if (a.dense) {
+    const int np = a.n / 256;
+    const int per_kvh = a.g * np;
+    const int bkv = int(x / per_kvh);
+    const int rest = int(x % per_kvh);
+    const int pair = np - 1 - rest / a.g;   // heavy units first
+    const int gi = rest % a.g;
+    u.b = bkv / a.Hkv; u.kvh = bkv % a.Hkv; u.h = u.kvh * a.g + gi;
+    u.q_tok = pair * 256;
+    u.n_past = 0; u.n_past_tiles = 0; u.last_cols = kTile;
+    u.c_tok = 0; u.n_cont = 2 * pair; u.d_tok = pair * 256;
+    u.seg_j = 0;
+  } else {
+    const int pp = a.seg / 256;
+    const int gi_p = a.g * pp;
+    const long long per_kvh = (long long)a.n1 * gi_p;
+    const int bkv = int(x / per_kvh);
+    const int rest = int(x % per_kvh);
+    const int j = a.n1 - 1 - rest / gi_p;
+    const int gi = (rest % gi_p) / pp;
+    const int p = rest % pp;
+    u.b = bkv / a.Hkv; u.kvh = bkv % a.Hkv; u.h = u.kvh * a.g + gi;
+    u.seg_j = j;
+    u.q_tok = j * a.seg + p * 256;
+    const long long unit = ((long long)u.b * a.Hq + u.h) * a.n1 + j;
+    u.list = a.idx + unit * a.k;
+    const int c = a.cnt[unit];
+    u.n_past = c - a.r;
+    u.ok = (c >= a.r) && (c <= a.k);
+    if (!u.ok) u.n_past = 0;
+    u.n_past_tiles = (u.n_past * a.blk + kTile - 1) / kTile;
+    u.last_cols = u.n_past * a.blk - (u.n_past_tiles - 1) * kTile;
+    u.c_tok = j * a.seg; u.n_cont = 2 * p; u.d_tok = u.q_tok;
+  }
+  u.T = u.n_past_tiles + u.n_cont + 2;
+  return u;
+}
+
+// ---------------------------------------------------------------- softmax role
+// mask kinds
+constexpr int kMaskNone = 0, kMaskCausal = 1, kMaskCols = 2;
+
+__device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars* bars, int which, int warp_in_wg,
+                                             int lane) {
+  const uint32_t tm = bars->tmem_base;
+  const uint32_t lane_off = uint32_t(warp_in_wg * 32) << 16;
+  const uint32_t tS = tm + lane_off + which * 128;
+  const uint32_t tO = tm + lane_off + 256 + which * 128;
+  const int row = warp_in_wg * 32 + lane;
+  const int my_tiles = which == 0 ? u.T - 1 : u.T;
+  const float c = a.sm_scale * 1.4426950408889634f;   // logits -> log2 units
+  float m_run = -CUDART_INF, l_run = 0.f;
+  bool alive = true;
+
+  for (int jt = 0; jt < my_tiles; ++jt) {
+    if (!mbar_wait(&bars->s_full[which], jt & 1, bars, a.st, 10 + which)) { alive = false; break; }
+    tc_fence_after();
+    uint32_t sv[128];
+    tmem_ld32(tS + 0, sv + 0);
+    tmem_ld32(tS + 32, sv + 32);
+    tmem_ld32(tS + 64, sv + 64);
+    tmem_ld32(tS + 96, sv + 96);
+    tmem_wait_ld();
+    float* s = reinterpret_cast<float*>(sv);
+
+    int kind = kMaskNone, cols = kTile;
+    if (jt == my_tiles - 1) kind = kMaskCausal;                                   // own diagonal tile
+    else if (jt == u.n_past_tiles - 1 && u.last_cols < kTile) { kind = kMaskCols; cols = u.last_cols; }
+    if (kind == kMaskCausal) {
+#pragma unroll
+      for (int i = 0; i < 128; ++i) s[i] = (i > row) ? -CUDART_INF : s[i];
+    } else if (kind == kMaskCols) {
+#pragma unroll
+      for (int i = 0; i < 128; ++i) s[i] = (i >= cols) ? -CUDART_INF : s[i];
+    }
+    float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
+#pragma unroll
+    for (int i = 4; i < 128; i += 4) {
+      mx0 = fmaxf(mx0, s[i]); mx1 = fmaxf(mx1, s[i + 1]); mx2 = fmaxf(mx2, s[i + 2]); mx3 = fmaxf(mx3, s[i + 3]);
+    }
+    const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+    const float m_new = fmaxf(m_run, m_tile);
+    // lazy rescale: keep the old reference maximum while the new one exceeds it by < 2^8
+    const bool need = (m_new - m_run) * c > kRescaleThreshold;   // true on the first tile (m_run = -inf)
+    if (jt == 0) {
+      m_run = m_new;
+    } else if (__any_sync(0xffffffffu, need)) {
+      const float f = need ? ex2((m_run - m_new) * c) : 1.f;
+      if (need) { m_run = m_new; l_run *= f; }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t ov[32];
+        tmem_ld32(tO + q * 32, ov);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
+        tmem_st32(tO + q * 32, ov);
+      }
+    }
+    const float neg_mc = -m_run * c;
+    float sum0 = 0.f, sum1 = 0.f;
+    uint32_t pk[64];
+#pragma unroll
+    for (int i = 0; i < 128; i += 2) {
+      const float p0 = ex2(fmaf(s[i], c, neg_mc));
+      const float p1 = ex2(fmaf(s[i + 1], c, neg_mc));
+      sum0 += p0; sum1 += p1;
+      pk[i >> 1] = pack_bf16(p0, p1);
+    }
+    l_run += sum0 + sum1;
+    tmem_st32(tS + 0, pk);
+    tmem_st32(tS + 32, pk + 32);
+    tmem_wait_st();
+    tc_fence_before();
+    mbar_arrive(&bars->p_full[which]);
+  }
+
+  if (alive && mbar_wait(&bars->o_done[which], 0, bars, a.st, 20 + which)) {
+    tc_fence_after();
+    const int t = u.q_tok + which * kTile + row;
+    __nv_bfloat16* orow = a.O + u.b * a.osb + u.h * a.osh + int64_t(t) * a.ost;
+    const float inv = 1.f / l_run;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t ov[32];
+      tmem_ld32(tO + q * 32, ov);
+      tmem_wait_ld();
+      uint4* dst = reinterpret_cast<uint4*>(orow + q * 32);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        uint4 w;
+        w.x = pack_bf16(__uint_as_float(ov[8 * i + 0]) * inv, __uint_as_float(ov[8 * i + 1]) * inv);
+        w.y = pack_bf16(__uint_as_float(ov[8 * i + 2]) * inv, __uint_as_float(ov[8 * i + 3]) * inv);
+        w.z = pack_bf16(__uint_as_float(ov[8 * i + 4]) * inv, __uint_as_float(ov[8 * i + 5]) * inv);
+        w.w = pack_bf16(__uint_as_float(ov[8 * i + 6]) * inv, __uint_as_float(ov[8 * i + 7]) * inv);
+        dst[i] = w;
+      }
+    }
+    if (a.lse != nullptr)
+      a.lse[((long long)u.b * a.Hq + u.h) * a.n + t] = m_run * a.sm_scale + __logf(l_run);
+  }
+}
+
+// ---------------------------------------------------------------- producer role
+__device__ __forceinline__ void producer_role(const Args& a, const Unit& u, Bars* bars, uint32_t smem_base,
+                                              const CUtensorMap* tmQ, const CUtensorMap* tmKb,
+                                              const CUtensorMap* tmVb, const CUtensorMap* tmKt,
+                                              const CUtensorMap* tmVt, int lane) {
+  if (lane == 0) {
+    mbar_expect_tx(&bars->q_full, 2 * kTileBytes);
+    for (int w = 0; w < 2; ++w)
+      for (int hf = 0; hf < 2; ++hf)
+        tma_load_4d(smem_base + kSmemQ + w * kTileBytes + hf * kHalfBytes, tmQ, &bars->q_full, hf * 64,
+                    u.q_tok + w * kTile, u.h, u.b);
+  }
+  const int bpt = kTile / a.blk;
+  for (int it = 0; it < 2 * u.T; ++it) {   // item 2*jt = K tile jt, item 2*jt+1 = V tile jt
+    const int slot = it % kSlots, use = it / kSlots;
+    if (use > 0 && !mbar_wait(&bars->kv_empty[slot], (use - 1) & 1, bars, a.st, 30)) return;
+    if (lane == 0) {
+      const int jt = it >> 1;
+      const bool is_v = it & 1;
+      const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
+      unsigned long long* bar = &bars->kv_full[slot];
+      mbar_expect_tx(bar, kTileBytes);
+      if (jt < u.n_past_tiles) {
+        const CUtensorMap* tm = is_v ? tmVb : tmKb;
+        for (int q = 0; q < bpt; ++q) {
+          const int li = jt * bpt + q;
+          // boxes beyond the list read past the end of the tensor and arrive as zeros
+          const int tok = li < u.n_past ? u.list[li] * a.blk : a.n;
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_4d(dst + hf * kHalfBytes + q * a.blk * 128, tm, bar, hf * 64, tok, u.kvh, u.b);
+        }
+      } else {
+        const CUtensorMap* tm = is_v ? tmVt : tmKt;
+        const int ci = jt - u.n_past_tiles;
+        const int tok = ci < u.n_cont ? u.c_tok + ci * kTile : u.d_tok + (ci - u.n_cont) * kTile;
+        for (int hf = 0; hf < 2; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, bar, hf * 64, tok, u.kvh, u.b);
+      }
+    }
+    __syncwarp();
+  }
+}
+
+// ---------------------------------------------------------------- MMA role
+__device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t q_smem, uint32_t k_smem) {
+  const uint64_t base = desc_base(16);
+#pragma unroll
+  for (int kk = 0; kk < kD / 16; ++kk) {
+    const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+    umma_ss(d_tmem, desc_at(base, q_smem + off), desc_at(base, k_smem + off), kIdescQK, kk > 0);
+  }
+}
+__device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint32_t v_smem, bool acc) {
+  const uint64_t base = desc_base(kHalfBytes);   // the two 64-column halves of head_dim are 16 KB apart
+#pragma unroll
+  for (int kk = 0; kk < kTile / 16; ++kk)
+    umma_ts(d_tmem, p_tmem + kk * 8, desc_at(base, v_smem + kk * 16 * 128), kIdescPV, (acc || kk > 0) ? 1u : 0u);
+}
+
+__device__ __forceinline__ void mma_role(const Args& a, const Unit& u, Bars* bars, uint32_t smem_base, int lane) {
+  const uint32_t tm = bars->tmem_base;
+  const uint32_t tS[2] = {tm, tm + 128}, tO[2] = {tm + 256, tm + 384};
+  const uint32_t qA = smem_base + kSmemQ, qB = qA + kTileBytes;
+  const int T = u.T, TA = u.T - 1;
+  auto slot_addr = [&](int item) { return smem_base + kSmemKV + (item % kSlots) * kTileBytes; };
+  auto full_wait = [&](int item) {
+    return mbar_wait(&bars->kv_full[item % kSlots], (item / kSlots) & 1, bars, a.st, 40);
+  };
+  if (!mbar_wait(&bars->q_full, 0, bars, a.st, 41)) return;
+  if (!full_wait(0)) return;
+  tc_fence_after();
+  if (lane == 0) {
+    issue_qk(tS[0], qA, slot_addr(0)); umma_commit(&bars->s_full[0]);
+    issue_qk(tS[1], qB, slot_addr(0)); umma_commit(&bars->s_full[1]);
+    umma_commit(&bars->kv_empty[0]);
+  }
+  __syncwarp();
+  for (int jt = 0; jt < T; ++jt) {
+    const bool has_next = jt + 1 < T;
+    if (has_next && !full_wait(2 * (jt + 1))) return;
+    if (!full_wait(2 * jt + 1)) return;
+    const uint32_t v_smem = slot_addr(2 * jt + 1);
+    const uint32_t kn_smem = slot_addr(2 * (jt + 1));
+    if (jt < TA) {
+      if (!mbar_wait(&bars->p_full[0], jt & 1, bars, a.st, 42)) return;
+      tc_fence_after();
+      if (lane == 0) {
+        issue_pv(tO[0], tS[0], v_smem, jt > 0);
+        if (jt + 1 < TA) { issue_qk(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
+        else umma_commit(&bars->o_done[0]);
+      }
+      __syncwarp();
+    }
+    if (!mbar_wait(&bars->p_full[1], jt & 1, bars, a.st, 43)) return;
+    tc_fence_after();
+    if (lane == 0) {
+      issue_pv(tO[1], tS[1], v_smem, jt > 0);
+      umma_commit(&bars->kv_empty[(2 * jt + 1) % kSlots]);
+      if (has_next) {
+        issue_qk(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
+        umma_commit(&bars->kv_empty[(2 * (jt + 1)) % kSlots]);
+      } else {
+        umma_commit(&bars->o_done[1]);
+      }
+    }
+    __syncwarp();
+  }
+}
+
+// ---------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kThreads, 1)
+attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKb,
+                       const __grid_constant__ CUtensorMap tmVb, const __grid_constant__ CUtensorMap tmKt,
+                       const __grid_constant__ CUtensorMap tmVt, const Args a) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t smem_base = (raw + 1023u) & ~1023u;
+  Bars* bars = reinterpret_cast<Bars*>(smem_raw + (smem_base - raw) + kSmemBar);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bars->q_full, 1);
+    for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->kv_full[i], 1); mbar_init(&bars->kv_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_full[i], 1); mbar_init(&bars->p_full[i], 128); mbar_init(&bars->o_done[i], 1); }
+    bars->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 8 && lane == 0) {
+    prefetch_tmap(&tmQ); prefetch_tmap(&tmKb); prefetch_tmap(&tmVb); prefetch_tmap(&tmKt); prefetch_tmap(&tmVt);
+  }
+  if (warp == 9) { tmem_alloc(&bars->tmem_base, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+
+  Unit u = decode_unit(a);
+  // the list contract: ascending past blocks, then exactly the r diagonal blocks
+  if (!a.dense) {
+    bool ok = u.ok;
+    if (ok) {
+      const int c = u.n_past + a.r;
+      for (int i = threadIdx.x; i < c; i += kThreads) {
+        const int v = u.list[i];
+        if (i >= u.n_past) ok = ok && (v == u.seg_j * a.r + (i - u.n_past));
+        else ok = ok && v >= 0 && v < u.seg_j * a.r && (i == 0 || u.list[i - 1] < v);
+      }
+    }
+    ok = __syncthreads_and(ok);
+    if (!ok && threadIdx.x == 0) report(a.st, CP_ERR_BOUNDS, 1, u.b, u.h, u.seg_j, u.n_past + a.r);
+    u.ok = ok;
+  }
+
+  if (u.ok) {
+    if (warp < 8) softmax_role(a, u, bars, warp >> 2, warp & 3, lane);
+    else if (warp == 8) producer_role(a, u, bars, smem_base, &tmQ, &tmKb, &tmVb, &tmKt, &tmVt, lane);
+    else mma_role(a, u, bars, smem_base, lane);
+  }
+  if (bars->abort_flag) {
+    // give copies and MMAs still in flight time to land before the CTA's resources go away
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) tmem_dealloc(bars->tmem_base, 512);
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [B, H, n, 128] bf16 with element strides (sb, sh, st); box = 64 columns x `rows` tokens
+bool make_map(CUtensorMap* map, const void* base, int B, int H, int n, const int64_t* s, int rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[4] = {cuuint64_t(kD), cuuint64_t(n), cuuint64_t(H), cuuint64_t(B)};
+  cuuint64_t strides[3] = {cuuint64_t(s[2]) * 2, cuuint64_t(s[1]) * 2, cuuint64_t(s[0]) * 2};
+  cuuint32_t box[4] = {64, cuuint32_t(rows), 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool sm100_path_applies(const cp_params& p, const Dims& m) {
+  return p.dtype == CP_BF16 && m.d == 128 && m.seg % 256 == 0 && (m.blk == 32 || m.blk == 64 || m.blk == 128) &&
+         !(p.flags & CP_FLAG_FORCE_SIMT);
+}
+
+int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, const void* K, const void* V,
+                           const int32_t* idx, const int32_t* cnt, void* O, float* lse, DeviceStatus* st,
+                           bool dense, cudaStream_t s) {
+  CUtensorMap tmQ, tmKb, tmVb, tmKt, tmVt;
+  if (!make_map(&tmQ, Q, m.B, m.Hq, m.n, p.q_stride, kTile) || !make_map(&tmKb, K, m.B, m.Hkv, m.n, p.k_stride, m.blk) ||
+      !make_map(&tmVb, V, m.B, m.Hkv, m.n, p.v_stride, m.blk) || !make_map(&tmKt, K, m.B, m.Hkv, m.n, p.k_stride, kTile) ||
+      !make_map(&tmVt, V, m.B, m.Hkv, m.n, p.v_stride, kTile))
+    return CP_ERR_CUDA;
+  Args a;
+  a.idx = idx; a.cnt = cnt; a.O = static_cast<__nv_bfloat16*>(O); a.lse = lse; a.st = st;
+  a.B = m.B; a.Hq = m.Hq; a.Hkv = m.Hkv; a.g = m.g; a.n = m.n; a.seg = m.seg; a.blk = m.blk; a.k = m.k;
+  a.r = m.r; a.n1 = m.n1;
+  a.osb = p.o_stride[0]; a.osh = p.o_stride[1]; a.ost = p.o_stride[2];
+  a.sm_scale = p.sm_scale; a.dense = dense ? 1 : 0;
+  const long long units = dense ? (long long)m.B * m.Hq * (m.n / 256) : (long long)m.B * m.Hq * m.n1 * (m.seg / 256);
+  if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
+  if (cudaFuncSetAttribute(attention_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)
+    return CP_ERR_CUDA;
+  attention_sm100_kernel<<<unsigned(units), kThreads, kSmemTotal, s>>>(tmQ, tmKb, tmVb, tmKt, tmVt, a);
+  return check_launch();
+}
+
+}  // namespace cp

@@ -1,0 +1,86 @@
+"""Shared helpers of the GPU parity tests: run the CUDA path through the C ABI and the fp64
+oracle on the same bits, and compare."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2409_12490_b200 import binding as cp
+
+TOL_BF16_MAX, TOL_BF16_MEAN = 1e-2, 1e-3     # attention, bf16 path (unit-scale inputs)
+TOL_F32 = 1e-5                               # attention, fp32 path
+EXCUSE_GAP = 1e-5                            # selection: k-th boundary gap (in ln S) below which a swap is excused
+
+
+def f32(x):
+    return np.float32(x).item()
+
+
+def problem(cfg, **kw):
+    return cp.Problem.from_config(cfg, **kw)
+
+
+def to_dev(*ts):
+    return [t.cuda() for t in ts]
+
+
+def oracle_scores(cfg, Q, K, S_prev=None, est_scale=None, mask_before_softmax=False):
+    return oracle.estimate(Q, K, cfg.segment_size, cfg.block_size,
+                           est_scale=f32(cfg.est_scale if est_scale is None else est_scale),
+                           alpha=f32(cfg.alpha), S_prev=S_prev, mask_before_softmax=mask_before_softmax)
+
+
+def compare_scores(S_gpu: torch.Tensor, S_ref: np.ndarray, atol=1e-9):
+    S = S_gpu.cpu().numpy()
+    assert S.shape == S_ref.shape
+    assert np.array_equal(np.isneginf(S), np.isneginf(S_ref)), "causal mask differs"
+    fin = np.isfinite(S_ref)
+    err = np.abs(S[fin] - S_ref[fin])
+    assert err.max() <= atol, f"ln S max abs err {err.max():.3e}"
+    return float(err.max())
+
+
+def compare_selection(idx_gpu, cnt_gpu, idx_ref, cnt_ref, S_ref, r):
+    """Sets must agree; a difference is excused only if every block in the symmetric difference
+    scores within EXCUSE_GAP of the oracle's last-admitted past score.  Returns (excused, unexcused)."""
+    ig, cg = idx_gpu.cpu().numpy(), cnt_gpu.cpu().numpy()
+    assert np.array_equal(cg, cnt_ref), "cnt differs"
+    excused = unexcused = 0
+    B, H, n1, k = idx_ref.shape
+    diff_units = np.argwhere((ig != idx_ref).any(-1))
+    for b, h, j in diff_units:
+        c = cnt_ref[b, h, j]
+        a, o = set(ig[b, h, j, :c].tolist()), set(idx_ref[b, h, j, :c].tolist())
+        if a == o:
+            unexcused += 1           # same set but order/padding differs: lists must be ascending
+            continue
+        past_o = [x for x in o if x < j * r]
+        thr = min(S_ref[b, h, j, x] for x in past_o)
+        ok = all(abs(S_ref[b, h, j, x] - thr) < EXCUSE_GAP for x in (a ^ o)) and len(a) == len(o)
+        excused += ok
+        unexcused += not ok
+    # every GPU list must be ascending and padded with -1
+    for b in range(B):
+        for h in range(H):
+            for j in range(n1):
+                c = cg[b, h, j]
+                row = ig[b, h, j]
+                assert (np.diff(row[:c]) > 0).all() and (row[c:] == -1).all()
+    return excused, unexcused
+
+
+def attention_errors(O_gpu: torch.Tensor, O_ref: np.ndarray):
+    err = np.abs(O_gpu.float().cpu().numpy().astype(np.float64) - O_ref)
+    return float(err.max()), float(err.mean())
+
+
+def sample_rows(cfg, n_units=16, seed=0, extra_rows=()):
+    """Rows (b,h,t) covering whole sampled (head, segment) units plus given single rows."""
+    rng = np.random.default_rng(seed)
+    rows = []
+    n1 = cfg.n1
+    m_seg = -(-(cfg.budget_blocks - cfg.r) // cfg.r)      # first segment with real selection
+    segs = sorted({0, min(1, n1 - 1), min(m_seg, n1 - 1), min(m_seg + 1, n1 - 1), n1 - 1})
+    units = [(0, int(rng.integers(cfg.n_q_heads)), s) for s in segs]
+    while len(units) < n_units:
+        units.append((int(rng.integers(cfg.batch)), int(rng.integers(cfg.n_q_heads)), int(rng.integers(n1))))
+    return units

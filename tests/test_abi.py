@@ -1,0 +1,43 @@
+"""The C-ABI library loads without a GPU and exports every symbol the header declares."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2409_12490_b200 import binding as cp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "critiprefill.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(critiprefill_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2409_12490_b200.build import build
+    build()
+    lib = cp.load_library()
+    names = declared_symbols()
+    assert set(cp.EXPORTS) <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_params_struct_size_matches_header_layout():
+    # 10 int32 + 12 int64 + 3 float + 1 int32
+    assert ctypes.sizeof(cp.CpParams) == 10 * 4 + 12 * 8 + 3 * 4 + 4
+
+
+def test_host_validation_without_gpu():
+    p = cp.Problem(1, 4, 2, 1024, 64, 128, 32, 8)
+    assert cp.workspace_bytes(p) > 256
+    with pytest.raises(cp.CritiPrefillError):
+        cp.workspace_bytes(cp.Problem(1, 4, 3, 1024, 64, 128, 32, 8))      # Hq % Hkv
+    with pytest.raises(cp.CritiPrefillError):
+        cp.workspace_bytes(cp.Problem(1, 4, 2, 1000, 64, 128, 32, 8))      # n % seg
+    with pytest.raises(cp.CritiPrefillError):
+        cp.workspace_bytes(cp.Problem(1, 4, 2, 1024, 64, 128, 32, 3))      # k < r
+    assert "workspace" in cp.status_string(4)
