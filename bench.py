@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the CritiPrefill prefill hot path on B200.
+
+One "step" is one pass of the whole path over one layer's Q/K/V:
+    critiprefill_estimate -> critiprefill_select -> critiprefill_attention
+on the 128K-token Llama3-8B-shaped workload (config C4), with inputs resident in HBM.
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C4] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2409_12490_b200 import CONFIGS  # noqa: E402
+from paper_2409_12490_b200.inputs import make_qkv  # noqa: E402
+
+METRIC = "128K prefill-attention ms (estimate+select+sparse attention, one layer)"
+# DRAM bytes per launch of the sparse attention kernel at the bench workload, from the ncu
+# capture summarised under profiles/ (None until one exists for the current kernel).
+ATTN_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "hbm_gbs": d["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def flop_counts(cfg):
+    """FLOPs per layer pass: what the sparse kernel executes (128x128 tiles, fully masked
+    diagonal tiles skipped), the causal-useful part, and dense causal attention."""
+    d, Hq, n, seg, blk, k, r, n1 = (cfg.head_dim, cfg.n_q_heads, cfg.seq_len, cfg.segment_size, cfg.block_size,
+                                    cfg.budget_blocks, cfg.r, cfg.n1)
+    tile = 4 * 128 * 128 * d                       # QK^T + PV for one 128x128 tile
+    q_tiles = seg // 128
+    executed = 0
+    listed = 0
+    for j in range(n1):
+        cnt = min(k, (j + 1) * r)
+        listed += cnt
+        past_tiles = -(-(cnt - r) * blk // 128)
+        for i in range(q_tiles):
+            executed += (past_tiles + i + 1) * tile
+    executed *= Hq * cfg.batch
+    full_tiles = 4 * seg * blk * d * Hq * listed * cfg.batch          # every listed block against the whole segment
+    useful = full_tiles - 4 * d * Hq * n1 * (seg * seg - seg * (seg + 1) // 2) * cfg.batch
+    dense = 4 * d * Hq * n * (n + 1) // 2 * cfg.batch
+    return {"executed": executed, "listed_full_tiles": full_tiles, "useful": useful, "dense": dense}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+        self.period = period_s
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+            nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+# ----------------------------------------------------------------------------- reference arm
+def oracle_step(cfg, Q, K, V, head, n_rows, seed):
+    """A bounded sample of one layer pass on the CPU oracle: Algorithm 1 + selection for one
+    query head, Algorithm 2 for `n_rows` random rows of it.  Returns (seconds_est_sel, seconds_attn)."""
+    import oracle
+    g = cfg.n_q_heads // cfg.n_kv_heads
+    q, k, v = Q[:, head:head + 1], K[:, head // g:head // g + 1], V[:, head // g:head // g + 1]
+    t0 = time.perf_counter()
+    S = oracle.estimate(q, k, cfg.segment_size, cfg.block_size, est_scale=cfg.est_scale, alpha=cfg.alpha)
+    idx, cnt = oracle.select(S, cfg.segment_size, cfg.block_size, cfg.budget_blocks)
+    t1 = time.perf_counter()
+    rng = np.random.default_rng(seed)
+    rows = np.stack([np.zeros(n_rows, np.int64), np.zeros(n_rows, np.int64),
+                     rng.integers(0, cfg.seq_len, n_rows)], axis=1)
+    oracle.sparse_attention_rows(q, k, v, idx, cnt, cfg.segment_size, cfg.block_size,
+                                 1.0 / math.sqrt(cfg.head_dim), rows)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def oracle_ms_per_layer(cfg, t_est, t_attn, n_rows):
+    """Extrapolate the sample to a whole layer pass by unit counts."""
+    total_rows = cfg.batch * cfg.n_q_heads * cfg.seq_len
+    return 1e3 * (t_est * cfg.n_q_heads * cfg.batch + t_attn * total_rows / n_rows)
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle.build
+    oracle.build.build()
+    Q, K, V = make_qkv(cfg)
+    n_rows = 256
+    cores = os.cpu_count()
+    for i in range(args.warmup):
+        oracle_step(cfg, Q, K, V, i % cfg.n_q_heads, n_rows, i)
+    ms = []
+    for i in range(args.steps):
+        te, ta = oracle_step(cfg, Q, K, V, (7 * i + 3) % cfg.n_q_heads, n_rows, 100 + i)
+        ms.append(oracle_ms_per_layer(cfg, te, ta, n_rows))
+    value = float(np.mean(ms))
+    sample = (f"per step: Algorithm 1 + selection for 1 of {cfg.n_q_heads} query heads (all segments) and "
+              f"Algorithm 2 for {n_rows} random rows of it; extrapolated to the layer by head and row counts")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "ms", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": value, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": value, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def workload_config(cfg):
+    return {"workload": f"{cfg.name}: 1 layer, batch {cfg.batch}, seq {cfg.seq_len}, {cfg.n_q_heads}Q/{cfg.n_kv_heads}KV "
+                        f"heads, head_dim {cfg.head_dim}, {cfg.dtype}, segment {cfg.segment_size}, block {cfg.block_size}, "
+                        f"budget {cfg.budget_tokens} tokens, est_scale {cfg.est_scale}, no layer fusion (first layer)",
+            "inputs": "seeded clustered-key / AR(1)-query generator", "l2": "inputs larger than L2 (Q alone "
+            f"{cfg.batch * cfg.n_q_heads * cfg.seq_len * cfg.head_dim * 2 / 1e6:.0f} MB vs 126 MB); no explicit flush"}
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    from paper_2409_12490_b200 import binding as cp
+    from paper_2409_12490_b200.build import build
+    if rank == 0:
+        build()
+    if dist is not None:
+        dist.barrier()
+    cp.load_library()
+
+    # every rank works on its own batch item (same shape, its own seed): weak scaling, no collective
+    Q, K, V = make_qkv(cfg, layer=rank)
+    hQ, hK, hV = Q.pin_memory(), K.pin_memory(), V.pin_memory()
+    dQ, dK, dV = hQ.to(dev, non_blocking=True), hK.to(dev, non_blocking=True), hV.to(dev, non_blocking=True)
+    prob = cp.Problem.from_config(cfg)
+    ws = cp.alloc_workspace(prob, dev)
+    S = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1, cfg.n2), dtype=torch.float64, device=dev)
+    idx = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1, cfg.budget_blocks), dtype=torch.int32, device=dev)
+    cnt = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1), dtype=torch.int32, device=dev)
+    O = torch.empty_like(dQ)
+    hO = torch.empty_like(hQ).pin_memory()
+    torch.cuda.synchronize()
+
+    def step(ev=None):
+        if ev is not None:
+            ev[0].record()
+        cp.estimate(prob, dQ, dK, ws, S_out=S)
+        if ev is not None:
+            ev[1].record()
+        cp.select(prob, S, ws, idx=idx, cnt=cnt)
+        if ev is not None:
+            ev[2].record()
+        cp.attention(prob, dQ, dK, dV, idx, cnt, ws, O=O)
+        if ev is not None:
+            ev[3].record()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(physical_gpu_index(local)) as clocks:
+        barrier()
+        start.record()
+        for i in range(args.steps):
+            step(evs[i])
+        end.record()
+        barrier()
+    total_ms = start.elapsed_time(end)
+    status = cp.device_status(ws)
+    if status != 0:
+        raise SystemExit(f"device status {status}: {cp.status_string(status)}")
+    est_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    sel_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    att_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    if dist is not None:
+        t = torch.tensor([total_ms, est_ms, sel_ms, att_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, est_ms, sel_ms, att_ms = t.tolist()
+    ms_per_step = total_ms / args.steps
+
+    # dense baseline of the same library (the denominator of the speed-up)
+    dense_ms = None
+    if not args.no_dense:
+        cp.dense_attention(prob, dQ, dK, dV, ws, O=O)
+        torch.cuda.synchronize()
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 2
+        d0.record()
+        for _ in range(reps):
+            cp.dense_attention(prob, dQ, dK, dV, ws, O=O)
+        d1.record()
+        torch.cuda.synchronize()
+        dense_ms = d0.elapsed_time(d1) / reps
+
+    # end to end through the public API with host buffers: H2D of Q,K,V, the path, D2H of O
+    e2e_steps = max(2, min(5, args.steps))
+    h2d = (hQ.numel() + hK.numel() + hV.numel()) * hQ.element_size()
+    d2h = hO.numel() * hO.element_size()
+
+    def e2e_step():
+        dQ.copy_(hQ, non_blocking=True); dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
+        step()
+        hO.copy_(O, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = t.item()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    fl = flop_counts(cfg)
+    achieved = fl["executed"] / (att_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "attention_sm100_kernel (critiprefill_attention)",
+                "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "peak_source": f"{peaks['source']} (burst)",
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
+                "flops_per_launch": fl["executed"], "traffic": ATTN_TRAFFIC_BYTES}
+    summary_bytes = (dQ.numel() + dK.numel()) * dQ.element_size()
+    out = {
+        "metric": METRIC, "value": ms_per_step, "unit": "ms", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": workload_config(cfg),
+        "breakdown_ms": {"estimate": est_ms, "select": sel_ms, "attention": att_ms},
+        "dense_ms": dense_ms,
+        "speedup_vs_dense": (dense_ms / ms_per_step) if dense_ms else None,
+        "dense_equiv_tflops": fl["dense"] / (ms_per_step * 1e-3) / 1e12,
+        "dense_kernel_tflops": (fl["dense"] / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
+        "estimate_gbs": summary_bytes / (est_ms * 1e-3) / 1e9,
+        "layer_passes_per_s": world * 1e3 / ms_per_step,
+        "paper_context": "paper: 2.7x (Llama3-8B) / 3.0x (Yi-9B) end-to-end prefill speed-up at 128K on one A100, fp16",
+        "roofline": roofline,
+        "e2e": {"value": e2e_ms, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": 4 * args.steps,
+        "clocks": clocks.summary(),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle.build
+        oracle.build.build()
+        n_rows = min(cfg.seq_len, 65536)
+        te, ta = oracle_step(cfg, Q, K, V, 5 % cfg.n_q_heads, n_rows, 0)
+        out["cpu_baseline"] = {
+            "value": oracle_ms_per_layer(cfg, te, ta, n_rows), "unit": "ms", "cores": os.cpu_count(), "kind": "oracle",
+            "sample": f"Algorithm 1 + selection for 1 of {cfg.n_q_heads} query heads ({te:.1f} s, numpy) and Algorithm 2 "
+                      f"for {n_rows} random rows ({ta:.1f} s, C/OpenMP); extrapolated to the layer by head and row counts"}
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="C4", choices=sorted(CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

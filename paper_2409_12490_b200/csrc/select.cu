@@ -13,6 +13,7 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 
 __device__ __forceinline__ unsigned long long ordered_key(double x) {
+  if (x == 0.0) x = 0.0;   // -0.0 and +0.0 compare equal and must map to one key
   unsigned long long u = (unsigned long long)__double_as_longlong(x);
   return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
 }
