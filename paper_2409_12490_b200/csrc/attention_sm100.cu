@@ -2,12 +2,12 @@
 // sm_100a tensor cores.  bf16 operands, fp32 accumulation in tensor memory, online softmax.
 //
 // One CTA works on 256 consecutive query rows of one (batch, query head): two 128-row tiles
-// "A" and "B" that share every K/V tile the producer brings in.  Roles (320 threads):
+// "A" and "B" that share every K/V tile the producer brings in.  Roles (384 threads):
 //   warps 0-3  softmax for tile A (one thread per query row)
 //   warps 4-7  softmax for tile B
 //   warp  8    TMA producer: K/V tiles through a 5-slot ring of 32 KB buffers; a gathered
 //              tile is assembled from 128/blk boxes addressed by the block list
-//   warp  9    MMA issuer: S = Q K^T (operands in shared memory), O += P V (P read from
+//   warp  9    MMA issuer (warps 10-11 idle; they complete the third warpgroup): S = Q K^T (operands in shared memory), O += P V (P read from
 //              tensor memory, where the softmax warps overwrite S with bf16 probabilities)
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each.
 // The tile sequence of a unit is: gathered past tiles, contiguous unmasked tiles, then the
@@ -26,7 +26,7 @@ constexpr int kTile = 128;
 constexpr int kHalfBytes = kTile * 64 * 2;   // [128 rows x 64 cols] bf16, 128-byte swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;   // both halves of head_dim
 constexpr int kSlots = 5;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
 constexpr int kSmemQ = 0;
 constexpr int kSmemKV = 2 * kTileBytes;
 constexpr int kSmemBar = kSmemKV + kSlots * kTileBytes;
@@ -160,6 +160,13 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -281,9 +288,11 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
     }
     float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
 #pragma unroll
-    for (int i = 4; i < 128; i += 4) {
-      mx0 = fmaxf(mx0, s[i]); mx1 = fmaxf(mx1, s[i + 1]); mx2 = fmaxf(mx2, s[i + 2]); mx3 = fmaxf(mx3, s[i + 3]);
+    for (int i = 4; i < 124; i += 8) {
+      mx0 = max3(mx0, s[i], s[i + 1]); mx1 = max3(mx1, s[i + 2], s[i + 3]);
+      mx2 = max3(mx2, s[i + 4], s[i + 5]); mx3 = max3(mx3, s[i + 6], s[i + 7]);
     }
+    mx0 = max3(mx0, s[124], s[125]); mx1 = max3(mx1, s[126], s[127]);
     const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
     const float m_new = fmaxf(m_run, m_tile);
     // lazy rescale: keep the old reference maximum while the new one exceeds it by < 2^8
@@ -304,15 +313,18 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
       }
     }
     const float neg_mc = -m_run * c;
-    float sum0 = 0.f, sum1 = 0.f;
+    const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
+    float2 sum2 = make_float2(0.f, 0.f);
     uint32_t pk[64];
 #pragma unroll
     for (int i = 0; i < 128; i += 2) {
-      const float p0 = ex2(fmaf(s[i], c, neg_mc));
-      const float p1 = ex2(fmaf(s[i + 1], c, neg_mc));
-      sum0 += p0; sum1 += p1;
-      pk[i >> 1] = pack_bf16(p0, p1);
+      const float2 x = __ffma2_rn(make_float2(s[i], s[i + 1]), c2, nm2);
+      float2 p;
+      p.x = ex2(x.x); p.y = ex2(x.y);
+      sum2 = __fadd2_rn(sum2, p);
+      pk[i >> 1] = pack_bf16(p.x, p.y);
     }
+    const float sum0 = sum2.x, sum1 = sum2.y;
     l_run += sum0 + sum1;
     tmem_st32(tS + 0, pk);
     tmem_st32(tS + 32, pk + 32);
@@ -483,6 +495,8 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   tc_fence_after();
 
   Unit u = decode_unit(a);
+  // once any CTA has reported a timeout the remaining CTAs do no work (keeps a broken run short)
+  if (a.st != nullptr && *reinterpret_cast<volatile int32_t*>(&a.st->code) == CP_ERR_TIMEOUT) u.ok = false;
   // the list contract: ascending past blocks, then exactly the r diagonal blocks
   if (!a.dense) {
     bool ok = u.ok;
@@ -499,10 +513,18 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     u.ok = ok;
   }
 
-  if (u.ok) {
-    if (warp < 8) softmax_role(a, u, bars, warp >> 2, warp & 3, lane);
-    else if (warp == 8) producer_role(a, u, bars, smem_base, &tmQ, &tmKb, &tmVb, &tmKt, &tmVt, lane);
-    else mma_role(a, u, bars, smem_base, lane);
+  // Register re-partition.  The pool is what the CTA was launched with (384 threads x 168):
+  // 256 x 224 + 128 x 56 = 64512 fits it exactly; asking for more would block forever.
+  static_assert(256 * 224 + 128 * 56 <= kThreads * 168, "setmaxnreg budget exceeds the launch allocation");
+  if (warp < 8) {
+    reg_inc<224>();
+    if (u.ok) softmax_role(a, u, bars, warp >> 2, warp & 3, lane);
+  } else {
+    reg_dec<56>();
+    if (u.ok) {
+      if (warp == 8) producer_role(a, u, bars, smem_base, &tmQ, &tmKb, &tmVb, &tmKt, &tmVt, lane);
+      else if (warp == 9) mma_role(a, u, bars, smem_base, lane);
+    }
   }
   if (bars->abort_flag) {
     // give copies and MMAs still in flight time to land before the CTA's resources go away

@@ -9,7 +9,7 @@
 namespace cp {
 
 constexpr int kStatusBytes = 256;   // head of the workspace: status word + diagnostics
-constexpr int kMaxBlocksN2 = 4096;  // estimate keeps 4*n2 fp64 logits in shared memory
+constexpr int kMaxBlocksN2 = 6144;  // estimate keeps 4*n2 fp64 logits per head in shared memory
 
 // Derived sizes of one problem.
 struct Dims {
