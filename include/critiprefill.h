@@ -47,7 +47,8 @@ typedef enum {
   CP_ERR_WORKSPACE = 4,   /* ws is NULL, misaligned (256 B) or smaller than workspace_bytes */
   CP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor-map encode) */
   CP_ERR_TIMEOUT = 6,     /* device: a bounded pipeline wait expired; outputs are invalid */
-  CP_ERR_BOUNDS = 7       /* device: a block list broke its contract; that segment was skipped */
+  CP_ERR_BOUNDS = 7,      /* device: a block list broke its contract; that segment was skipped */
+  CP_ERR_STATIC_LIMIT = 8 /* critiprefill_estimate_static: problem needs more scratch than the built-in array holds */
 } cp_status;
 
 typedef enum { CP_BF16 = 0, CP_F32 = 1 } cp_dtype;
@@ -88,6 +89,29 @@ int critiprefill_workspace_bytes(const cp_params* p, size_t* bytes_out);
  * Arithmetic: fp64 on the representatives (which are exact in the input dtype). */
 int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, const double* S_prev,
                           double* S_out, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* critiprefill_estimate for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of this library, not part of the method.)
+ * Meant for code that cannot obtain a workspace where it calls us -- a server whose memory
+ * pool took the whole device at start-up, a loop that must not incur cudaMalloc's device-wide
+ * synchronisation, a plug-in bound by its host's allocation rules.  Same arguments, results
+ * and arithmetic as critiprefill_estimate, minus `ws`: the summaries go to an 8 MiB array
+ * that is part of the library's device image (critiprefill_static_scratch_bytes(); every GPU
+ * that loads the library holds it until the process exits).
+ *   - Problems whose critiprefill_workspace_bytes exceeds that size return
+ *     CP_ERR_STATIC_LIMIT and launch nothing.
+ *   - The call allocates and frees nothing (no cudaMalloc/cudaFree, no allocating library
+ *     routine).  The first call on each device resolves the array's device address with
+ *     cudaGetSymbolAddress (that device must be current); make that first call during
+ *     set-up, before any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents;
+ *     the library clears the part that must start at zero.  Two calls whose kernels overlap
+ *     on the GPU (different streams, no ordering between them) race on it: serialise them. */
+int critiprefill_estimate_static(const cp_params* p, const void* Q, const void* K, const double* S_prev,
+                                 double* S_out, void* cuda_stream);
+
+/* Size in bytes of the built-in scratch array used by critiprefill_estimate_static. */
+size_t critiprefill_static_scratch_bytes(void);
 
 /* Algorithm 2, line 8: I_j = argtop_k(S[j], k) with the diagonal blocks always kept.
  *   S    in   device, [B,Hq,n1,n2] fp64 (as written by critiprefill_estimate)

@@ -24,6 +24,7 @@ FLAG_FORCE_SIMT = 2
 EXPORTS = (
     "critiprefill_workspace_bytes", "critiprefill_estimate", "critiprefill_select",
     "critiprefill_attention", "critiprefill_dense_attention", "critiprefill_device_status",
+    "critiprefill_estimate_static", "critiprefill_static_scratch_bytes",
     "critiprefill_status_string",
 )
 
@@ -66,10 +67,13 @@ def load_library() -> ctypes.CDLL:
         lib.critiprefill_attention.argtypes = [PP, P, P, P, P, P, P, P, P, SZ, P]
         lib.critiprefill_dense_attention.argtypes = [PP, P, P, P, P, P, P, SZ, P]
         lib.critiprefill_device_status.argtypes = [P, ctypes.POINTER(ctypes.c_int32), P]
+        lib.critiprefill_estimate_static.argtypes = [PP, P, P, P, P, P]
+        lib.critiprefill_static_scratch_bytes.argtypes = []
         lib.critiprefill_status_string.argtypes = [ctypes.c_int]
         lib.critiprefill_status_string.restype = ctypes.c_char_p
         for name in EXPORTS[:-1]:
             getattr(lib, name).restype = ctypes.c_int
+        lib.critiprefill_static_scratch_bytes.restype = ctypes.c_size_t
         _lib = lib
     return _lib
 
@@ -168,6 +172,21 @@ def estimate(prob: Problem, Q, K, ws, S_prev=None, S_out=None) -> torch.Tensor:
     _check(load_library().critiprefill_estimate(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(S_prev), _ptr(S_out),
                                                 _ptr(ws), ws.numel(), _stream()), "critiprefill_estimate")
     return S_out
+
+
+def estimate_static(prob: Problem, Q, K, S_prev=None, S_out=None) -> torch.Tensor:
+    """critiprefill_estimate_static: critiprefill_estimate without a caller workspace, for callers
+    that cannot allocate device memory (the scratch is a fixed array inside the library)."""
+    if S_out is None:
+        S_out = torch.empty((prob.batch, prob.n_q_heads, prob.n1, prob.n2), dtype=torch.float64, device=Q.device)
+    p = prob.params(Q=Q, K=K)
+    _check(load_library().critiprefill_estimate_static(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(S_prev), _ptr(S_out),
+                                                       _stream()), "critiprefill_estimate_static")
+    return S_out
+
+
+def static_scratch_bytes() -> int:
+    return int(load_library().critiprefill_static_scratch_bytes())
 
 
 def select(prob: Problem, S, ws, idx=None, cnt=None):

@@ -116,6 +116,7 @@ const char* critiprefill_status_string(int status) {
     case CP_ERR_CUDA: return "a CUDA call failed";
     case CP_ERR_TIMEOUT: return "device: a bounded pipeline wait expired";
     case CP_ERR_BOUNDS: return "device: a block list broke its contract";
+    case CP_ERR_STATIC_LIMIT: return "problem needs more scratch than the library's built-in static array holds";
     default: return "unknown status";
   }
 }
