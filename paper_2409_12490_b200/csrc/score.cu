@@ -12,7 +12,7 @@
 namespace cp {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
 
 template <typename T> __device__ __forceinline__ double to_f64(T x);
@@ -69,7 +69,7 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
     double acc[U][4];
 #pragma unroll
     for (int u = 0; u < U; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.0;
-#pragma unroll 2
+#pragma unroll 4
     for (int v = 0; v < D / VE; ++v) {
       const uint4 a = __ldg(pmx + v), c = __ldg(pmn + v);
       const T* ka = reinterpret_cast<const T*>(&a);
