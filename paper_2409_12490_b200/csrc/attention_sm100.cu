@@ -41,6 +41,9 @@ struct Bars {
   unsigned long long s_full[2];
   unsigned long long p_full[2];
   unsigned long long o_done[2];
+#ifdef CP_TRACE
+  unsigned long long dbg;
+#endif
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -56,6 +59,14 @@ struct Args {
   float sm_scale;
   int dense;
 };
+
+// Optional cycle trace (compiled only with -DCP_TRACE, never in the product build): one CTA
+// records clock64() stamps into the workspace behind the status block.
+#ifdef CP_TRACE
+#define CP_STAMP(cond, slot) do { if (cond) reinterpret_cast<long long*>(reinterpret_cast<char*>(a.st) + 256)[slot] = clock64(); } while (0)
+#else
+#define CP_STAMP(cond, slot) do { } while (0)
+#endif
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -120,20 +131,28 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+// The MMA and commit wrappers are executed by ALL lanes of the issuing warp with warp-uniform
+// operands (so descriptors live in uniform registers); elect.sync inside picks the one lane
+// that actually issues.
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      "{\n.reg .pred p, e;\n.reg .b32 lid;\nelect.sync lid|e, 0xffffffff;\nsetp.ne.b32 p, %4, 0;\n"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
   asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      "{\n.reg .pred p, e;\n.reg .b32 lid;\nelect.sync lid|e, 0xffffffff;\nsetp.ne.b32 p, %4, 0;\n"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+  asm volatile(
+      "{\n.reg .pred e;\n.reg .b32 lid;\nelect.sync lid|e, 0xffffffff;\n"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}"
+      ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
   asm volatile(
@@ -266,7 +285,10 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
   bool alive = true;
 
   for (int jt = 0; jt < my_tiles; ++jt) {
+    const bool tr = blockIdx.x == 0 && warp_in_wg == 0 && lane == 0 && jt < 64;
+    CP_STAMP(tr, which * 1024 + jt * 8 + 0);
     if (!mbar_wait(&bars->s_full[which], jt & 1, bars, a.st, 10 + which)) { alive = false; break; }
+    CP_STAMP(tr, which * 1024 + jt * 8 + 1);
     tc_fence_after();
     uint32_t sv[128];
     tmem_ld32(tS + 0, sv + 0);
@@ -274,6 +296,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
     tmem_ld32(tS + 64, sv + 64);
     tmem_ld32(tS + 96, sv + 96);
     tmem_wait_ld();
+    CP_STAMP(tr, which * 1024 + jt * 8 + 2);
     float* s = reinterpret_cast<float*>(sv);
 
     int kind = kMaskNone, cols = kTile;
@@ -312,6 +335,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
         tmem_st32(tO + q * 32, ov);
       }
     }
+    CP_STAMP(tr, which * 1024 + jt * 8 + 3);
     const float neg_mc = -m_run * c;
     const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
     float2 sum2 = make_float2(0.f, 0.f);
@@ -326,11 +350,13 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
     }
     const float sum0 = sum2.x, sum1 = sum2.y;
     l_run += sum0 + sum1;
+    CP_STAMP(tr, which * 1024 + jt * 8 + 4);
     tmem_st32(tS + 0, pk);
     tmem_st32(tS + 32, pk + 32);
     tmem_wait_st();
     tc_fence_before();
     mbar_arrive(&bars->p_full[which]);
+    CP_STAMP(tr, which * 1024 + jt * 8 + 5);
   }
 
   if (alive && mbar_wait(&bars->o_done[which], 0, bars, a.st, 20 + which)) {
@@ -418,7 +444,7 @@ __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint3
 }
 
 __device__ __forceinline__ void mma_role(const Args& a, const Unit& u, Bars* bars, uint32_t smem_base, int lane) {
-  const uint32_t tm = bars->tmem_base;
+  const uint32_t tm = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
   const uint32_t tS[2] = {tm, tm + 128}, tO[2] = {tm + 256, tm + 384};
   const uint32_t qA = smem_base + kSmemQ, qB = qA + kTileBytes;
   const int T = u.T, TA = u.T - 1;
@@ -429,41 +455,75 @@ __device__ __forceinline__ void mma_role(const Args& a, const Unit& u, Bars* bar
   if (!mbar_wait(&bars->q_full, 0, bars, a.st, 41)) return;
   if (!full_wait(0)) return;
   tc_fence_after();
-  if (lane == 0) {
-    issue_qk(tS[0], qA, slot_addr(0)); umma_commit(&bars->s_full[0]);
-    issue_qk(tS[1], qB, slot_addr(0)); umma_commit(&bars->s_full[1]);
-    umma_commit(&bars->kv_empty[0]);
+#ifdef CP_TRACE
+  if (blockIdx.x == 0) {
+    // MMA throughput probes: 64 back-to-back instructions of each kind into scratch accumulators
+    long long* tb = reinterpret_cast<long long*>(reinterpret_cast<char*>(a.st) + 256) + 3000;
+    for (int kind = 0; kind < 4; ++kind) {
+      const long long t0 = clock64();
+      {
+        for (int rep = 0; rep < 8; ++rep) {
+          if (kind == 0) issue_qk(tS[0], qA, slot_addr(0));                 // SS, N=128
+          else if (kind == 1) issue_pv(tO[0], tS[1], slot_addr(0), true);   // TS, N=128
+          else if (kind == 2) {                                             // SS, N=64
+            const uint64_t base = desc_base(16);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+              umma_ss(tS[0], desc_at(base, qA + off), desc_at(base, slot_addr(0) + off), idesc, 1);
+            }
+          } else {                                                          // SS, N=256 (rows run on into the next buffer)
+            const uint64_t base = desc_base(16);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+            for (int kk = 0; kk < 8; ++kk) {
+              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
+              umma_ss(tS[0], desc_at(base, qA + off), desc_at(base, qA + off), idesc, 1);
+            }
+          }
+        }
+        umma_commit(&bars->dbg);
+      }
+      __syncwarp();
+      const long long t1 = clock64();
+      mbar_wait(&bars->dbg, kind & 1, bars, a.st, 99);
+      const long long t2 = clock64();
+      if (lane == 0) { tb[kind * 2] = t1 - t0; tb[kind * 2 + 1] = t2 - t0; }
+    }
+    tc_fence_after();
   }
-  __syncwarp();
+#endif
+  issue_qk(tS[0], qA, slot_addr(0)); umma_commit(&bars->s_full[0]);
+  issue_qk(tS[1], qB, slot_addr(0)); umma_commit(&bars->s_full[1]);
+  umma_commit(&bars->kv_empty[0]);
   for (int jt = 0; jt < T; ++jt) {
     const bool has_next = jt + 1 < T;
     if (has_next && !full_wait(2 * (jt + 1))) return;
     if (!full_wait(2 * jt + 1)) return;
     const uint32_t v_smem = slot_addr(2 * jt + 1);
     const uint32_t kn_smem = slot_addr(2 * (jt + 1));
+    const bool tr = blockIdx.x == 0 && lane == 0 && jt < 64;
+    CP_STAMP(tr, 2048 + jt * 8 + 0);
     if (jt < TA) {
       if (!mbar_wait(&bars->p_full[0], jt & 1, bars, a.st, 42)) return;
+      CP_STAMP(tr, 2048 + jt * 8 + 1);
       tc_fence_after();
-      if (lane == 0) {
-        issue_pv(tO[0], tS[0], v_smem, jt > 0);
-        if (jt + 1 < TA) { issue_qk(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
-        else umma_commit(&bars->o_done[0]);
-      }
-      __syncwarp();
+      issue_pv(tO[0], tS[0], v_smem, jt > 0);
+      if (jt + 1 < TA) { issue_qk(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
+      else umma_commit(&bars->o_done[0]);
     }
+    CP_STAMP(tr, 2048 + jt * 8 + 2);
     if (!mbar_wait(&bars->p_full[1], jt & 1, bars, a.st, 43)) return;
+    CP_STAMP(tr, 2048 + jt * 8 + 3);
     tc_fence_after();
-    if (lane == 0) {
-      issue_pv(tO[1], tS[1], v_smem, jt > 0);
-      umma_commit(&bars->kv_empty[(2 * jt + 1) % kSlots]);
-      if (has_next) {
-        issue_qk(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
-        umma_commit(&bars->kv_empty[(2 * (jt + 1)) % kSlots]);
-      } else {
-        umma_commit(&bars->o_done[1]);
-      }
+    issue_pv(tO[1], tS[1], v_smem, jt > 0);
+    umma_commit(&bars->kv_empty[(2 * jt + 1) % kSlots]);
+    if (has_next) {
+      issue_qk(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
+      umma_commit(&bars->kv_empty[(2 * (jt + 1)) % kSlots]);
+    } else {
+      umma_commit(&bars->o_done[1]);
     }
-    __syncwarp();
+    CP_STAMP(tr, 2048 + jt * 8 + 4);
   }
 }
 
@@ -482,6 +542,9 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     mbar_init(&bars->q_full, 1);
     for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->kv_full[i], 1); mbar_init(&bars->kv_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_full[i], 1); mbar_init(&bars->p_full[i], 128); mbar_init(&bars->o_done[i], 1); }
+#ifdef CP_TRACE
+    mbar_init(&bars->dbg, 1);
+#endif
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
