@@ -19,13 +19,16 @@ template <typename T> __device__ __forceinline__ double to_f64(T x);
 template <> __device__ __forceinline__ double to_f64<float>(float x) { return double(x); }
 template <> __device__ __forceinline__ double to_f64<__nv_bfloat16>(__nv_bfloat16 x) { return double(__bfloat162float(x)); }
 
+// ln(e^a + e^b).  When the smaller term is more than e^-50 below the larger one it cannot change
+// the rounded result (|hi| is at most a few hundred here), so the transcendental pair is skipped.
 __device__ __forceinline__ double logaddexp(double a, double b) {
   const double hi = fmax(a, b), lo = fmin(a, b);
-  if (hi == -CUDART_INF) return -CUDART_INF;
-  return hi + log1p(exp(lo - hi));
+  const double d = lo - hi;                 // <= 0, or NaN when both are -inf
+  if (!(d > -50.0)) return hi;
+  return hi + log1p(exp(d));
 }
 
-// Shared memory: q[U][D] as (max, min) pairs, then logits lg[U][4][n2].
+// Shared memory: logits lg[U][4][n2].
 template <typename T, int D, int U>
 __global__ void __launch_bounds__(kThreads)
 score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __restrict__ Kmax,
@@ -33,9 +36,7 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
              int Hq, int g, int n1, int n2, int seg, int blk, double est_scale, double ln_alpha,
              double ln_1m_alpha, int fuse, int mask_first) {
   extern __shared__ double smem[];
-  double2* q2 = reinterpret_cast<double2*>(smem);   // [U][D]: .x = Qmax, .y = Qmin
-  double* lg = smem + 2 * U * D;                    // [U][4][n2]
-  __shared__ double red[4 * U][kWarps];
+  double* lg = smem;                                // [U][4][n2]
   __shared__ double stat[4 * U];
 
   // CTA -> (b, kv head, head subgroup, segment)
@@ -50,116 +51,112 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   auto unit_of = [&](int u) { return (size_t(b) * Hq + h0 + u) * n1 + j; };
 
-  for (int i = tid; i < U * D; i += kThreads) {
-    const int u = i / D, c = i % D;
-    const size_t off = unit_of(u) * D + c;
-    q2[i] = make_double2(to_f64(Qmax[off]), to_f64(Qmin[off]));
-  }
-  __syncthreads();
-
   // blocks that start at or after the end of the segment are masked (line 13)
   const int visible = min(n2, ((j + 1) * seg + blk - 1) / blk);
   const T* kmx_base = Kmax + size_t(kvh) * n2 * D;
   const T* kmn_base = Kmin + size_t(kvh) * n2 * D;
-  constexpr int VE = 16 / sizeof(T);   // elements per 16-byte load
 
-  for (int bb = tid; bb < n2; bb += kThreads) {
-    const uint4* pmx = reinterpret_cast<const uint4*>(kmx_base + size_t(bb) * D);
-    const uint4* pmn = reinterpret_cast<const uint4*>(kmn_base + size_t(bb) * D);
-    double acc[U][4];
+  // The 8 x n2 x D logit products run on the fp64 tensor-core path (mma.m8n8k4): the 8 rows of
+  // A are (head u, representative) = (u0 max, u0 min, u1 max, ...); B columns are key blocks.
+  // Lane l supplies A[l/4][l%4] and B[l%4][l/4] per k-step and owns C[l/4][2(l%4)+{0,1}].
+  // The channel order inside the dot product is free, so lane-in-quad q takes the D/4
+  // contiguous channels [q*D/4, (q+1)*D/4): one contiguous slice of a summary row per lane.
+  constexpr int KS = D / 4;                 // k-steps
+  constexpr int VE = 16 / sizeof(T);        // elements per 16-byte load
+  constexpr int NV = KS / VE;               // 16-byte loads per lane per row
+  const int quad = lane & 3, grp = lane >> 2;
+  double afrag[KS];
+  {
+    const int u = grp >> 1, rep = grp & 1;
+    const T* src = (rep == 0 ? Qmax : Qmin) + (u < U ? unit_of(u) : unit_of(0)) * D + quad * KS;
 #pragma unroll
-    for (int u = 0; u < U; ++u) acc[u][0] = acc[u][1] = acc[u][2] = acc[u][3] = 0.0;
-#pragma unroll 4
-    for (int v = 0; v < D / VE; ++v) {
-      const uint4 a = __ldg(pmx + v), c = __ldg(pmn + v);
-      const T* ka = reinterpret_cast<const T*>(&a);
-      const T* kc = reinterpret_cast<const T*>(&c);
-      double kx[VE], kn[VE];
+    for (int ks = 0; ks < KS; ++ks) afrag[ks] = u < U ? to_f64(src[ks]) : 0.0;
+  }
+  const int n_tiles = (n2 + 7) / 8;
+  for (int t = warp; t < n_tiles; t += kWarps) {
+    const int bblk = min(t * 8 + grp, n2 - 1);          // this lane's B column (clamped in a ragged last tile)
+    const uint4* pmx = reinterpret_cast<const uint4*>(kmx_base + size_t(bblk) * D + quad * KS);
+    const uint4* pmn = reinterpret_cast<const uint4*>(kmn_base + size_t(bblk) * D + quad * KS);
+    uint4 vx[NV], vn[NV];
 #pragma unroll
-      for (int e = 0; e < VE; ++e) { kx[e] = to_f64(ka[e]); kn[e] = to_f64(kc[e]); }
+    for (int v = 0; v < NV; ++v) { vx[v] = __ldg(pmx + v); vn[v] = __ldg(pmn + v); }
+    double cx0 = 0.0, cx1 = 0.0, cn0 = 0.0, cn1 = 0.0;
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
+    for (int v = 0; v < NV; ++v) {
+      const T* ka = reinterpret_cast<const T*>(&vx[v]);
+      const T* kc = reinterpret_cast<const T*>(&vn[v]);
 #pragma unroll
-        for (int e = 0; e < VE; ++e) {
-          const double2 q = q2[u * D + v * VE + e];
-          acc[u][0] = fma(q.x, kx[e], acc[u][0]); acc[u][1] = fma(q.x, kn[e], acc[u][1]);
-          acc[u][2] = fma(q.y, kx[e], acc[u][2]); acc[u][3] = fma(q.y, kn[e], acc[u][3]);
+      for (int e = 0; e < VE; ++e) {
+        const double a = afrag[v * VE + e];
+        const double bx = to_f64(ka[e]), bn = to_f64(kc[e]);
+        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                     : "+d"(cx0), "+d"(cx1) : "d"(a), "d"(bx));
+        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                     : "+d"(cn0), "+d"(cn1) : "d"(a), "d"(bn));
+      }
+    }
+    // C rows: grp = (u, rep); rep 0 (Qmax): cx = l1, cn = l2; rep 1 (Qmin): cx = l3, cn = l4
+    const int u = grp >> 1, rep = grp & 1;
+    if (u < U) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int bb = t * 8 + quad * 2 + i;
+        if (bb < n2) {
+          const bool hide = mask_first && bb >= visible;
+          lg[(u * 4 + rep * 2 + 0) * n2 + bb] = hide ? -CUDART_INF : (i ? cx1 : cx0) * est_scale;
+          lg[(u * 4 + rep * 2 + 1) * n2 + bb] = hide ? -CUDART_INF : (i ? cn1 : cn0) * est_scale;
         }
       }
     }
-    const bool hide = mask_first && bb >= visible;
-#pragma unroll
-    for (int u = 0; u < U; ++u)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) lg[(u * 4 + i) * n2 + bb] = hide ? -CUDART_INF : acc[u][i] * est_scale;
   }
   __syncthreads();
 
-  // log-sum-exp of each of the 4U logit rows (softmax over blocks, lines 9-10): max, then sum
-  double part[4 * U];
-#pragma unroll
-  for (int rI = 0; rI < 4 * U; ++rI) {
+  // log-sum-exp of each of the 4U logit rows (softmax over blocks, lines 9-10): a warp owns a
+  // row, so only shuffles are needed; terms more than e^-50 below the maximum are skipped
+#pragma unroll 1
+  for (int rI = warp; rI < 4 * U; rI += kWarps) {
+    const double* rowp = lg + rI * n2;
     double m = -CUDART_INF;
-    for (int bb = tid; bb < n2; bb += kThreads) m = fmax(m, lg[rI * n2 + bb]);
+    for (int bb = lane; bb < n2; bb += 32) m = fmax(m, rowp[bb]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (lane == 0) red[rI][warp] = m;
-  }
-  __syncthreads();
-  if (tid < 4 * U) {
-    double m = red[tid][0];
-    for (int w = 1; w < kWarps; ++w) m = fmax(m, red[tid][w]);
-    stat[tid] = m;
-  }
-  __syncthreads();
-#pragma unroll
-  for (int rI = 0; rI < 4 * U; ++rI) {
-    const double m = stat[rI];
     double sum = 0.0;
-    for (int bb = tid; bb < n2; bb += kThreads) sum += exp(lg[rI * n2 + bb] - m);
+#pragma unroll 4
+    for (int bb = lane; bb < n2; bb += 32) {
+      const double d = rowp[bb] - m;
+      if (d > -50.0) sum += exp(d);
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    part[rI] = sum;
-  }
-  __syncthreads();   // red[] is reused
-#pragma unroll
-  for (int rI = 0; rI < 4 * U; ++rI)
-    if (lane == 0) red[rI][warp] = part[rI];
-  __syncthreads();
-  if (tid < 4 * U) {
-    double sum = 0.0;
-    for (int w = 0; w < kWarps; ++w) sum += red[tid][w];
-    stat[tid] = stat[tid] + log(sum);
+    if (lane == 0) stat[rI] = m + log(sum);
   }
   __syncthreads();
 
+  // combine (lines 11-12), mask (13), fusion (14) over the U rows of this CTA, flattened
   const double ln2 = 0.693147180559945309417232121458;
-#pragma unroll
-  for (int u = 0; u < U; ++u) {
-    const double e1 = stat[u * 4 + 0], e2 = stat[u * 4 + 1], e3 = stat[u * 4 + 2], e4 = stat[u * 4 + 3];
-    double* out = S_out + unit_of(u) * n2;
-    const double* prev = fuse ? S_prev + unit_of(u) * n2 : nullptr;
-    const double* l = lg + u * 4 * n2;
-    for (int bb = tid; bb < n2; bb += kThreads) {
-      double v;
-      if (bb >= visible) {
-        v = -CUDART_INF;
-      } else {
-        const double L1 = l[bb] - e1, L2 = l[n2 + bb] - e2, L3 = l[2 * n2 + bb] - e3, L4 = l[3 * n2 + bb] - e4;
-        const double Lmax = logaddexp(L1, L3) - ln2;   // ln (S1+S3)/2
-        const double Lmin = logaddexp(L2, L4) - ln2;   // ln (S2+S4)/2
-        v = fmax(Lmax, Lmin);
-        if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + prev[bb]);
-      }
-      out[bb] = v;
+#pragma unroll 2
+  for (int e = tid; e < U * n2; e += kThreads) {
+    const int u = e / n2, bb = e - u * n2;
+    double v;
+    if (bb >= visible) {
+      v = -CUDART_INF;
+    } else {
+      const double* l = lg + u * 4 * n2;
+      const double L1 = l[bb] - stat[u * 4 + 0], L2 = l[n2 + bb] - stat[u * 4 + 1];
+      const double L3 = l[2 * n2 + bb] - stat[u * 4 + 2], L4 = l[3 * n2 + bb] - stat[u * 4 + 3];
+      const double Lmax = logaddexp(L1, L3) - ln2;   // ln (S1+S3)/2
+      const double Lmin = logaddexp(L2, L4) - ln2;   // ln (S2+S4)/2
+      v = fmax(Lmax, Lmin);
+      if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + S_prev[unit_of(u) * n2 + bb]);
     }
+    S_out[unit_of(u) * n2 + bb] = v;
   }
 }
 
 template <typename T, int D, int U>
 int launch_u(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
              double est_scale, double alpha, int fuse, int mask_first, cudaStream_t st) {
-  const size_t smem = sizeof(double) * (2 * size_t(U) * D + 4 * size_t(U) * m.n2);
+  const size_t smem = sizeof(double) * (4 * size_t(U) * m.n2);
   auto kern = score_kernel<T, D, U>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
     return CP_ERR_CUDA;
@@ -177,7 +174,7 @@ int launch_t(const Dims& m, const char* ws, const WsLayout& w, const double* S_p
              double est_scale, double alpha, int fuse, int mask_first, cudaStream_t st) {
   // as many heads per CTA as divide the group and keep the logits within ~200 KB of shared memory
   const size_t budget = 200 * 1024;
-  auto fits = [&](int U) { return m.g % U == 0 && sizeof(double) * (2 * size_t(U) * D + 4 * size_t(U) * m.n2) <= budget; };
+  auto fits = [&](int U) { return m.g % U == 0 && sizeof(double) * (4 * size_t(U) * m.n2) <= budget; };
   if (fits(4)) return launch_u<T, D, 4>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, st);
   if (fits(2)) return launch_u<T, D, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, st);
   if (fits(1)) return launch_u<T, D, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, st);
