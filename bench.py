@@ -26,6 +26,7 @@ sys.path.insert(0, ROOT)
 
 from paper_2409_12490_b200 import CONFIGS  # noqa: E402
 from paper_2409_12490_b200.inputs import make_qkv  # noqa: E402
+from paper_2409_12490_b200.sharding import RankInfo, aggregate_time_metric, layer_seed_for_rank, max_over_ranks  # noqa: E402
 
 METRIC = "128K prefill-attention ms (estimate+select+sparse attention, one layer)"
 # DRAM bytes per launch of the sparse attention kernel at the bench workload, from the ncu
@@ -186,16 +187,16 @@ def run_reference(args, cfg):
 def workload_config(cfg):
     return {"workload": f"{cfg.name}: 1 layer, batch {cfg.batch}, seq {cfg.seq_len}, {cfg.n_q_heads}Q/{cfg.n_kv_heads}KV "
                         f"heads, head_dim {cfg.head_dim}, {cfg.dtype}, segment {cfg.segment_size}, block {cfg.block_size}, "
-                        f"budget {cfg.budget_tokens} tokens, est_scale {cfg.est_scale}, no layer fusion (first layer)",
+                        f"budget {cfg.budget_tokens} tokens, est_scale {cfg.est_scale}, "
+                        + (f"{cfg.layers}-layer stack with layer fusion alpha {cfg.alpha}" if cfg.layers > 1 else "no layer fusion (first layer)"),
             "inputs": "seeded clustered-key / AR(1)-query generator", "l2": "inputs larger than L2 (Q alone "
             f"{cfg.batch * cfg.n_q_heads * cfg.seq_len * cfg.head_dim * 2 / 1e6:.0f} MB vs 126 MB); no explicit flush"}
 
 
 # ----------------------------------------------------------------------------- our arm
 def run_ours(args, cfg):
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    info = RankInfo.from_env()
+    rank, world, local = info.rank, info.world, info.local_rank
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -214,13 +215,23 @@ def run_ours(args, cfg):
         dist.barrier()
     cp.load_library()
 
-    # every rank works on its own batch item (same shape, its own seed): weak scaling, no collective
-    Q, K, V = make_qkv(cfg, layer=rank)
+    # every rank works on its own batch item (same shape, its own seed): weak scaling, no collective.
+    # A stack of L layers cycles through D distinct seeded layer inputs; the criticality scores are
+    # carried from layer to layer (Algorithm 1, line 14) through two ping-pong buffers.
+    L = args.layers if args.layers else cfg.layers
+    D = min(L, args.distinct_layers)
+    layers_in = []
+    for li in range(D):
+        q, k, v = make_qkv(cfg, layer=layer_seed_for_rank(li, rank, D))
+        if li == 0:
+            Q, K, V = q, k, v
+        layers_in.append(tuple(t.to(dev) for t in (q, k, v)))
     hQ, hK, hV = Q.pin_memory(), K.pin_memory(), V.pin_memory()
-    dQ, dK, dV = hQ.to(dev, non_blocking=True), hK.to(dev, non_blocking=True), hV.to(dev, non_blocking=True)
+    dQ, dK, dV = layers_in[0]
     prob = cp.Problem.from_config(cfg)
     ws = cp.alloc_workspace(prob, dev)
     S = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1, cfg.n2), dtype=torch.float64, device=dev)
+    S2 = torch.empty_like(S) if L > 1 else None
     idx = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1, cfg.budget_blocks), dtype=torch.int32, device=dev)
     cnt = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1), dtype=torch.int32, device=dev)
     O = torch.empty_like(dQ)
@@ -228,17 +239,31 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
 
     def step(ev=None):
+        """One pass of the whole path over the stack (L = 1: one layer)."""
+        if L == 1:
+            if ev is not None:
+                ev[0].record()
+            cp.estimate(prob, dQ, dK, ws, S_out=S)
+            if ev is not None:
+                ev[1].record()
+            cp.select(prob, S, ws, idx=idx, cnt=cnt)
+            if ev is not None:
+                ev[2].record()
+            cp.attention(prob, dQ, dK, dV, idx, cnt, ws, O=O)
+            if ev is not None:
+                ev[3].record()
+            return
         if ev is not None:
             ev[0].record()
-        cp.estimate(prob, dQ, dK, ws, S_out=S)
+        prev, cur = None, S
+        for li in range(L):
+            q, k, v = layers_in[li % D]
+            cp.estimate(prob, q, k, ws, S_prev=prev, S_out=cur)
+            cp.select(prob, cur, ws, idx=idx, cnt=cnt)
+            cp.attention(prob, q, k, v, idx, cnt, ws, O=O)
+            prev, cur = cur, (S2 if cur is S else S)
         if ev is not None:
-            ev[1].record()
-        cp.select(prob, S, ws, idx=idx, cnt=cnt)
-        if ev is not None:
-            ev[2].record()
-        cp.attention(prob, dQ, dK, dV, idx, cnt, ws, O=O)
-        if ev is not None:
-            ev[3].record()
+            ev[1].record(); ev[2].record(); ev[3].record()
 
     def barrier():
         torch.cuda.synchronize()
@@ -265,11 +290,9 @@ def run_ours(args, cfg):
     est_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
     sel_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     att_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
-    if dist is not None:
-        t = torch.tensor([total_ms, est_ms, sel_ms, att_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, est_ms, sel_ms, att_ms = t.tolist()
-    ms_per_step = total_ms / args.steps
+    total_ms, est_ms, sel_ms, att_ms = max_over_ranks([total_ms, est_ms, sel_ms, att_ms], dist, dev)
+    agg = aggregate_time_metric(total_ms / args.steps / L, world)      # per layer pass
+    ms_per_step = agg["ms_per_step"]
 
     # dense baseline of the same library (the denominator of the speed-up)
     dense_ms = None
@@ -291,8 +314,11 @@ def run_ours(args, cfg):
     d2h = hO.numel() * hO.element_size()
 
     def e2e_step():
+        """Host buffers in, host buffer out, one layer through the public API."""
         dQ.copy_(hQ, non_blocking=True); dK.copy_(hK, non_blocking=True); dV.copy_(hV, non_blocking=True)
-        step()
+        cp.estimate(prob, dQ, dK, ws, S_out=S)
+        cp.select(prob, S, ws, idx=idx, cnt=cnt)
+        cp.attention(prob, dQ, dK, dV, idx, cnt, ws, O=O)
         hO.copy_(O, non_blocking=True)
 
     e2e_step()
@@ -304,10 +330,7 @@ def run_ours(args, cfg):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = t.item()
+    (e2e_ms,) = max_over_ranks([e2e_ms], dist, dev)
 
     if rank != 0:
         if dist is not None:
@@ -316,6 +339,14 @@ def run_ours(args, cfg):
 
     peaks = load_peaks()
     fl = flop_counts(cfg)
+    if L > 1:   # the stack run has no per-kernel events: time the attention kernel alone
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(5):
+            cp.attention(prob, dQ, dK, dV, idx, cnt, ws, O=O)
+        a1.record()
+        torch.cuda.synchronize()
+        att_ms, est_ms, sel_ms = a0.elapsed_time(a1) / 5, None, None
     achieved = fl["executed"] / (att_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "attention_sm100_kernel (critiprefill_attention)",
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -333,12 +364,13 @@ def run_ours(args, cfg):
         "speedup_vs_dense": (dense_ms / ms_per_step) if dense_ms else None,
         "dense_equiv_tflops": fl["dense"] / (ms_per_step * 1e-3) / 1e12,
         "dense_kernel_tflops": (fl["dense"] / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
-        "estimate_gbs": summary_bytes / (est_ms * 1e-3) / 1e9,
-        "layer_passes_per_s": world * 1e3 / ms_per_step,
+        "estimate_gbs": (summary_bytes / (est_ms * 1e-3) / 1e9) if est_ms else None,
+        "layer_passes_per_s": agg["layer_passes_per_s"],
+        "layers": L, "distinct_layer_inputs": D, "stack_ms": ms_per_step * L,
         "paper_context": "paper: 2.7x (Llama3-8B) / 3.0x (Yi-9B) end-to-end prefill speed-up at 128K on one A100, fp16",
         "roofline": roofline,
         "e2e": {"value": e2e_ms, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": 4 * args.steps,
+        "gpu_launches": 4 * args.steps * L,
         "clocks": clocks.summary(),
     }
     if world == 1 and not args.no_cpu_baseline:
@@ -355,6 +387,54 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_sweep(args, cfg):
+    """Accuracy-vs-speed trace: budget x block size, each against the dense kernel.  Mass recall is
+    exp(lse_sparse - lse_dense), the share of a row's dense softmax mass that its listed keys hold."""
+    from paper_2409_12490_b200 import binding as cp
+    from paper_2409_12490_b200.build import build
+    build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    Q, K, V = (t.to(dev) for t in make_qkv(cfg))
+    rows = []
+    dense = None
+    for blk in (32, 64, 128):
+        for budget in (1024, 2048, 4096, 8192):
+            c = cfg.with_(block_size=blk, budget_tokens=budget)
+            prob = cp.Problem.from_config(c)
+            ws = cp.alloc_workspace(prob, dev)
+            if dense is None:
+                Od, lsed = cp.dense_attention(prob, Q, K, V, ws, want_lse=True)
+                torch.cuda.synchronize()
+                d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                d0.record()
+                cp.dense_attention(prob, Q, K, V, ws, O=Od, lse=lsed)
+                d1.record()
+                torch.cuda.synchronize()
+                dense = d0.elapsed_time(d1)
+            for _ in range(3):
+                O, S, idx, cnt = cp.prefill_layer(prob, Q, K, V, ws)
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            reps = 5
+            e[0].record()
+            for _ in range(reps):
+                S = cp.estimate(prob, Q, K, ws, S_out=S)
+                cp.select(prob, S, ws, idx=idx, cnt=cnt)
+                cp.attention(prob, Q, K, V, idx, cnt, ws, O=O)
+            e[1].record()
+            torch.cuda.synchronize()
+            ms = e[0].elapsed_time(e[1]) / reps
+            _, lse = cp.attention(prob, Q, K, V, idx, cnt, ws, O=O, want_lse=True)
+            assert cp.device_status(ws) == 0
+            recall = torch.exp(lse.double() - lsed.double())
+            diff = (O.float() - Od.float()).abs()
+            rows.append({"block": blk, "budget_tokens": budget, "ms": ms, "speedup_vs_dense": dense / ms,
+                         "mass_recall_mean": recall.mean().item(), "mass_recall_median": recall.median().item(),
+                         "mass_recall_p05": recall.flatten().kthvalue(max(1, recall.numel() // 20)).values.item(),
+                         "out_vs_dense_max": diff.max().item(), "out_vs_dense_mean": diff.mean().item()})
+    print(json.dumps({"sweep": rows, "dense_ms": dense, "config": workload_config(cfg), "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -362,12 +442,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="C4", choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=0, help="layers in the stack (default: the config's)")
+    ap.add_argument("--distinct-layers", type=int, default=2, help="distinct seeded layer inputs cycled through a stack")
+    ap.add_argument("--sweep", action="store_true", help="budget x block-size sweep (accuracy vs speed) instead of the bench line")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
     if args.impl == "reference":
         run_reference(args, cfg)
+    elif args.sweep:
+        run_sweep(args, cfg)
     else:
         run_ours(args, cfg)
 
