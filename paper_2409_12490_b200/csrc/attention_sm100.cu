@@ -1,8 +1,8 @@
 // K4 / K5: block-sparse (Algorithm 2, lines 6-13) and dense causal (Eq. 2) attention on the
 // sm_100a tensor cores.  bf16 operands, fp32 accumulation in tensor memory, online softmax.
 //
-// One CTA works on 256 consecutive query rows of one (batch, query head): two 128-row tiles
-// "A" and "B" that share every K/V tile the producer brings in.  Roles (384 threads):
+// Persistent CTAs (one per SM) walk over work units; a unit is 256 consecutive query rows of one
+// (batch, query head): two 128-row tiles "A" and "B" that share every K/V tile the producer brings in.  Roles (384 threads):
 //   warps 0-3  softmax for tile A (one thread per query row)
 //   warps 4-7  softmax for tile B
 //   warp  8    TMA producer: K/V tiles through a 5-slot ring of 32 KB buffers; a gathered
@@ -36,14 +36,15 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct Bars {
   unsigned long long q_full;
+  unsigned long long q_empty;
   unsigned long long kv_full[kSlots];
   unsigned long long kv_empty[kSlots];
   unsigned long long s_full[2];
   unsigned long long p_full[2];
   unsigned long long o_done[2];
-#ifdef CP_TRACE
-  unsigned long long dbg;
-#endif
+  unsigned long long sched_full[2];
+  unsigned long long sched_empty[2];
+  int sched_unit[2];
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -58,6 +59,8 @@ struct Args {
   int64_t osb, osh, ost;
   float sm_scale;
   int dense;
+  int n_units;
+  unsigned int* work_counter;   // next unit to hand out (zeroed by the host before the launch)
 };
 
 // Optional cycle trace (compiled only with -DCP_TRACE, never in the product build): one CTA
@@ -222,20 +225,21 @@ struct Unit {
   int T;            // tiles for B; A takes T-1
   const int32_t* list;
   int seg_j;
-  bool ok;
+  int cnt;
 };
 
-__device__ __forceinline__ Unit decode_unit(const Args& a) {
+// Units are ordered KV-head-major so that CTAs resident at the same time share K/V tiles in
+// L2; within a KV head the dense kernel takes the longest rows first.
+__device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
   Unit u;
-  u.ok = true;
   u.list = nullptr;
-  long long x = blockIdx.x;
+  u.cnt = 0;
   if (a.dense) {
     const int np = a.n / 256;
     const int per_kvh = a.g * np;
-    const int bkv = int(x / per_kvh);
-    const int rest = int(x % per_kvh);
-    const int pair = np - 1 - rest / a.g;   // heavy units first
+    const int bkv = x / per_kvh;
+    const int rest = x - bkv * per_kvh;
+    const int pair = np - 1 - rest / a.g;
     const int gi = rest % a.g;
     u.b = bkv / a.Hkv; u.kvh = bkv % a.Hkv; u.h = u.kvh * a.g + gi;
     u.q_tok = pair * 256;
@@ -245,9 +249,9 @@ __device__ __forceinline__ Unit decode_unit(const Args& a) {
   } else {
     const int pp = a.seg / 256;
     const int gi_p = a.g * pp;
-    const long long per_kvh = (long long)a.n1 * gi_p;
-    const int bkv = int(x / per_kvh);
-    const int rest = int(x % per_kvh);
+    const int per_kvh = a.n1 * gi_p;
+    const int bkv = x / per_kvh;
+    const int rest = x - bkv * per_kvh;
     const int j = a.n1 - 1 - rest / gi_p;
     const int gi = (rest % gi_p) / pp;
     const int p = rest % pp;
@@ -256,10 +260,8 @@ __device__ __forceinline__ Unit decode_unit(const Args& a) {
     u.q_tok = j * a.seg + p * 256;
     const long long unit = ((long long)u.b * a.Hq + u.h) * a.n1 + j;
     u.list = a.idx + unit * a.k;
-    const int c = a.cnt[unit];
-    u.n_past = c - a.r;
-    u.ok = (c >= a.r) && (c <= a.k);
-    if (!u.ok) u.n_past = 0;
+    u.cnt = a.cnt[unit];
+    u.n_past = min(max(u.cnt - a.r, 0), a.k);
     u.n_past_tiles = (u.n_past * a.blk + kTile - 1) / kTile;
     u.last_cols = u.n_past * a.blk - (u.n_past_tiles - 1) * kTile;
     u.c_tok = j * a.seg; u.n_cont = 2 * p; u.d_tok = u.q_tok;
@@ -268,98 +270,152 @@ __device__ __forceinline__ Unit decode_unit(const Args& a) {
   return u;
 }
 
+// The list contract, checked by every warp for itself (all warps reach the same verdict, so
+// no CTA-wide synchronisation is needed): r <= cnt <= k, ascending past blocks, then exactly
+// the r diagonal blocks of the segment.
+__device__ __forceinline__ bool unit_ok(const Args& a, const Unit& u, int lane) {
+  if (a.dense) return true;
+  bool ok = (u.cnt >= a.r) && (u.cnt <= a.k);
+  if (ok) {
+    for (int i = lane; i < u.cnt; i += 32) {
+      const int v = u.list[i];
+      if (i >= u.n_past) ok = ok && (v == u.seg_j * a.r + (i - u.n_past));
+      else ok = ok && v >= 0 && v < u.seg_j * a.r && (i == 0 || u.list[i - 1] < v);
+    }
+  }
+  return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ bool stop_requested(const Args& a, Bars* bars) {
+  return bars->abort_flag || (a.st != nullptr && *reinterpret_cast<volatile int32_t*>(&a.st->code) == CP_ERR_TIMEOUT);
+}
+
+// ---------------------------------------------------------------- unit scheduler
+// Units are handed out dynamically (an atomic counter in global memory) so that SMs that run
+// faster take more of them.  The producer warp draws the q-th unit of this CTA and publishes
+// it through a two-entry ring; the MMA warp and the eight softmax warps read it from there.
+__device__ __forceinline__ int publish_unit(const Args& a, Bars* bars, uint32_t q, int lane, bool* ok) {
+  const uint32_t slot = q & 1;
+  *ok = true;
+  if (q >= 2 && !mbar_wait(&bars->sched_empty[slot], ((q >> 1) - 1) & 1, bars, a.st, 50)) { *ok = false; return 0; }
+  int x = 0;
+  if (lane == 0) {
+    x = int(min(atomicAdd(a.work_counter, 1u), 0x7fffffffu));
+    bars->sched_unit[slot] = x;
+    mbar_arrive(&bars->sched_full[slot]);
+  }
+  return __shfl_sync(0xffffffffu, x, 0);
+}
+__device__ __forceinline__ int receive_unit(const Args& a, Bars* bars, uint32_t q, int lane, bool* ok) {
+  const uint32_t slot = q & 1;
+  *ok = mbar_wait(&bars->sched_full[slot], (q >> 1) & 1, bars, a.st, 51);
+  if (!*ok) return 0;
+  const int x = *reinterpret_cast<volatile int*>(&bars->sched_unit[slot]);
+  __syncwarp();
+  if (lane == 0) mbar_arrive(&bars->sched_empty[slot]);
+  return x;
+}
+
 // ---------------------------------------------------------------- softmax role
-// mask kinds
 constexpr int kMaskNone = 0, kMaskCausal = 1, kMaskCols = 2;
 
-__device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars* bars, int which, int warp_in_wg,
-                                             int lane) {
+__device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int which, int warp_in_wg, int lane) {
   const uint32_t tm = bars->tmem_base;
   const uint32_t lane_off = uint32_t(warp_in_wg * 32) << 16;
   const uint32_t tS = tm + lane_off + which * 128;
   const uint32_t tO = tm + lane_off + 256 + which * 128;
   const int row = warp_in_wg * 32 + lane;
-  const int my_tiles = which == 0 ? u.T - 1 : u.T;
   const float c = a.sm_scale * 1.4426950408889634f;   // logits -> log2 units
-  float m_run = -CUDART_INF, l_run = 0.f;
-  bool alive = true;
+  uint32_t n_tiles = 0;                               // S tiles consumed so far (all units)
+  uint32_t n_units = 0;                               // units finished so far
 
-  for (int jt = 0; jt < my_tiles; ++jt) {
-    const bool tr = blockIdx.x == 0 && warp_in_wg == 0 && lane == 0 && jt < 64;
-    CP_STAMP(tr, which * 1024 + jt * 8 + 0);
-    if (!mbar_wait(&bars->s_full[which], jt & 1, bars, a.st, 10 + which)) { alive = false; break; }
-    CP_STAMP(tr, which * 1024 + jt * 8 + 1);
-    tc_fence_after();
-    uint32_t sv[128];
-    tmem_ld32(tS + 0, sv + 0);
-    tmem_ld32(tS + 32, sv + 32);
-    tmem_ld32(tS + 64, sv + 64);
-    tmem_ld32(tS + 96, sv + 96);
-    tmem_wait_ld();
-    CP_STAMP(tr, which * 1024 + jt * 8 + 2);
-    float* s = reinterpret_cast<float*>(sv);
+  for (uint32_t q = 0;; ++q) {
+    bool got;
+    const int x = receive_unit(a, bars, q, lane, &got);
+    if (!got || x >= a.n_units || stop_requested(a, bars)) return;
+    const Unit u = decode_unit(a, x);
+    if (!unit_ok(a, u, lane)) continue;
+    const int my_tiles = which == 0 ? u.T - 1 : u.T;
+    float m_run = -CUDART_INF, l_run = 0.f;
 
-    int kind = kMaskNone, cols = kTile;
-    if (jt == my_tiles - 1) kind = kMaskCausal;                                   // own diagonal tile
-    else if (jt == u.n_past_tiles - 1 && u.last_cols < kTile) { kind = kMaskCols; cols = u.last_cols; }
-    if (kind == kMaskCausal) {
+    for (int jt = 0; jt < my_tiles; ++jt, ++n_tiles) {
+      const bool tr = blockIdx.x == 0 && q == 0 && warp_in_wg == 0 && lane == 0 && jt < 64;
+      CP_STAMP(tr, which * 1024 + jt * 8 + 0);
+      if (!mbar_wait(&bars->s_full[which], n_tiles & 1, bars, a.st, 10 + which)) return;
+      CP_STAMP(tr, which * 1024 + jt * 8 + 1);
+      tc_fence_after();
+      uint32_t sv[128];
+      tmem_ld32(tS + 0, sv + 0);
+      tmem_ld32(tS + 32, sv + 32);
+      tmem_ld32(tS + 64, sv + 64);
+      tmem_ld32(tS + 96, sv + 96);
+      tmem_wait_ld();
+      CP_STAMP(tr, which * 1024 + jt * 8 + 2);
+      float* s = reinterpret_cast<float*>(sv);
+
+      int kind = kMaskNone, cols = kTile;
+      if (jt == my_tiles - 1) kind = kMaskCausal;                                   // own diagonal tile
+      else if (jt == u.n_past_tiles - 1 && u.last_cols < kTile) { kind = kMaskCols; cols = u.last_cols; }
+      if (kind == kMaskCausal) {
 #pragma unroll
-      for (int i = 0; i < 128; ++i) s[i] = (i > row) ? -CUDART_INF : s[i];
-    } else if (kind == kMaskCols) {
+        for (int i = 0; i < 128; ++i) s[i] = (i > row) ? -CUDART_INF : s[i];
+      } else if (kind == kMaskCols) {
 #pragma unroll
-      for (int i = 0; i < 128; ++i) s[i] = (i >= cols) ? -CUDART_INF : s[i];
-    }
-    float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
-#pragma unroll
-    for (int i = 4; i < 124; i += 8) {
-      mx0 = max3(mx0, s[i], s[i + 1]); mx1 = max3(mx1, s[i + 2], s[i + 3]);
-      mx2 = max3(mx2, s[i + 4], s[i + 5]); mx3 = max3(mx3, s[i + 6], s[i + 7]);
-    }
-    mx0 = max3(mx0, s[124], s[125]); mx1 = max3(mx1, s[126], s[127]);
-    const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-    const float m_new = fmaxf(m_run, m_tile);
-    // lazy rescale: keep the old reference maximum while the new one exceeds it by < 2^8
-    const bool need = (m_new - m_run) * c > kRescaleThreshold;   // true on the first tile (m_run = -inf)
-    if (jt == 0) {
-      m_run = m_new;
-    } else if (__any_sync(0xffffffffu, need)) {
-      const float f = need ? ex2((m_run - m_new) * c) : 1.f;
-      if (need) { m_run = m_new; l_run *= f; }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t ov[32];
-        tmem_ld32(tO + q * 32, ov);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
-        tmem_st32(tO + q * 32, ov);
+        for (int i = 0; i < 128; ++i) s[i] = (i >= cols) ? -CUDART_INF : s[i];
       }
-    }
-    CP_STAMP(tr, which * 1024 + jt * 8 + 3);
-    const float neg_mc = -m_run * c;
-    const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
-    float2 sum2 = make_float2(0.f, 0.f);
-    uint32_t pk[64];
+      float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
 #pragma unroll
-    for (int i = 0; i < 128; i += 2) {
-      const float2 x = __ffma2_rn(make_float2(s[i], s[i + 1]), c2, nm2);
-      float2 p;
-      p.x = ex2(x.x); p.y = ex2(x.y);
-      sum2 = __fadd2_rn(sum2, p);
-      pk[i >> 1] = pack_bf16(p.x, p.y);
+      for (int i = 4; i < 124; i += 8) {
+        mx0 = max3(mx0, s[i], s[i + 1]); mx1 = max3(mx1, s[i + 2], s[i + 3]);
+        mx2 = max3(mx2, s[i + 4], s[i + 5]); mx3 = max3(mx3, s[i + 6], s[i + 7]);
+      }
+      mx0 = max3(mx0, s[124], s[125]); mx1 = max3(mx1, s[126], s[127]);
+      const float m_tile = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      const float m_new = fmaxf(m_run, m_tile);
+      // lazy rescale: keep the old reference maximum while the new one exceeds it by < 2^8
+      const bool need = (m_new - m_run) * c > kRescaleThreshold;   // true on the first tile (m_run = -inf)
+      if (jt == 0) {
+        m_run = m_new;
+      } else if (__any_sync(0xffffffffu, need)) {
+        const float f = need ? ex2((m_run - m_new) * c) : 1.f;
+        if (need) { m_run = m_new; l_run *= f; }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t ov[32];
+          tmem_ld32(tO + q * 32, ov);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
+          tmem_st32(tO + q * 32, ov);
+        }
+      }
+      CP_STAMP(tr, which * 1024 + jt * 8 + 3);
+      const float neg_mc = -m_run * c;
+      const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
+      float2 sum2 = make_float2(0.f, 0.f);
+      uint32_t pk[64];
+#pragma unroll
+      for (int i = 0; i < 128; i += 2) {
+        const float2 xx = __ffma2_rn(make_float2(s[i], s[i + 1]), c2, nm2);
+        float2 p;
+        p.x = ex2(xx.x); p.y = ex2(xx.y);
+        sum2 = __fadd2_rn(sum2, p);
+        pk[i >> 1] = pack_bf16(p.x, p.y);
+      }
+      l_run += sum2.x + sum2.y;
+      CP_STAMP(tr, which * 1024 + jt * 8 + 4);
+      tmem_st32(tS + 0, pk);
+      tmem_st32(tS + 32, pk + 32);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->p_full[which]);
+      CP_STAMP(tr, which * 1024 + jt * 8 + 5);
     }
-    const float sum0 = sum2.x, sum1 = sum2.y;
-    l_run += sum0 + sum1;
-    CP_STAMP(tr, which * 1024 + jt * 8 + 4);
-    tmem_st32(tS + 0, pk);
-    tmem_st32(tS + 32, pk + 32);
-    tmem_wait_st();
-    tc_fence_before();
-    mbar_arrive(&bars->p_full[which]);
-    CP_STAMP(tr, which * 1024 + jt * 8 + 5);
-  }
 
-  if (alive && mbar_wait(&bars->o_done[which], 0, bars, a.st, 20 + which)) {
+    // epilogue: O / l -> bf16 -> global.  The next unit's first PV cannot start before this
+    // thread signals its next P, so O is not overwritten while it is being read.
+    if (!mbar_wait(&bars->o_done[which], n_units & 1, bars, a.st, 20 + which)) return;
+    ++n_units;
     tc_fence_after();
     const int t = u.q_tok + which * kTile + row;
     __nv_bfloat16* orow = a.O + u.b * a.osb + u.h * a.osh + int64_t(t) * a.ost;
@@ -386,44 +442,58 @@ __device__ __forceinline__ void softmax_role(const Args& a, const Unit& u, Bars*
 }
 
 // ---------------------------------------------------------------- producer role
-__device__ __forceinline__ void producer_role(const Args& a, const Unit& u, Bars* bars, uint32_t smem_base,
-                                              const CUtensorMap* tmQ, const CUtensorMap* tmKb,
-                                              const CUtensorMap* tmVb, const CUtensorMap* tmKt,
-                                              const CUtensorMap* tmVt, int lane) {
-  if (lane == 0) {
-    mbar_expect_tx(&bars->q_full, 2 * kTileBytes);
-    for (int w = 0; w < 2; ++w)
-      for (int hf = 0; hf < 2; ++hf)
-        tma_load_4d(smem_base + kSmemQ + w * kTileBytes + hf * kHalfBytes, tmQ, &bars->q_full, hf * 64,
-                    u.q_tok + w * kTile, u.h, u.b);
-  }
+__device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_t smem_base, const CUtensorMap* tmQ,
+                                              const CUtensorMap* tmKb, const CUtensorMap* tmVb,
+                                              const CUtensorMap* tmKt, const CUtensorMap* tmVt, int lane) {
   const int bpt = kTile / a.blk;
-  for (int it = 0; it < 2 * u.T; ++it) {   // item 2*jt = K tile jt, item 2*jt+1 = V tile jt
-    const int slot = it % kSlots, use = it / kSlots;
-    if (use > 0 && !mbar_wait(&bars->kv_empty[slot], (use - 1) & 1, bars, a.st, 30)) return;
-    if (lane == 0) {
-      const int jt = it >> 1;
-      const bool is_v = it & 1;
-      const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
-      unsigned long long* bar = &bars->kv_full[slot];
-      mbar_expect_tx(bar, kTileBytes);
-      if (jt < u.n_past_tiles) {
-        const CUtensorMap* tm = is_v ? tmVb : tmKb;
-        for (int q = 0; q < bpt; ++q) {
-          const int li = jt * bpt + q;
-          // boxes beyond the list read past the end of the tensor and arrive as zeros
-          const int tok = li < u.n_past ? u.list[li] * a.blk : a.n;
-          for (int hf = 0; hf < 2; ++hf)
-            tma_load_4d(dst + hf * kHalfBytes + q * a.blk * 128, tm, bar, hf * 64, tok, u.kvh, u.b);
-        }
-      } else {
-        const CUtensorMap* tm = is_v ? tmVt : tmKt;
-        const int ci = jt - u.n_past_tiles;
-        const int tok = ci < u.n_cont ? u.c_tok + ci * kTile : u.d_tok + (ci - u.n_cont) * kTile;
-        for (int hf = 0; hf < 2; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, bar, hf * 64, tok, u.kvh, u.b);
-      }
+  uint32_t item = 0;      // K/V tiles issued so far (all units): item i lives in slot i % kSlots
+  uint32_t n_units = 0;
+  for (uint32_t q = 0;; ++q) {
+    bool got;
+    const int x = publish_unit(a, bars, q, lane, &got);
+    if (!got || x >= a.n_units || stop_requested(a, bars)) return;
+    const Unit u = decode_unit(a, x);
+    if (!unit_ok(a, u, lane)) {
+      if (lane == 0) report(a.st, CP_ERR_BOUNDS, 1, u.b, u.h, u.seg_j, u.cnt);
+      continue;
     }
-    __syncwarp();
+    // Q tiles: the buffer is free once every QK^T of the previous unit has completed
+    if (n_units > 0 && !mbar_wait(&bars->q_empty, (n_units - 1) & 1, bars, a.st, 31)) return;
+    if (lane == 0) {
+      mbar_expect_tx(&bars->q_full, 2 * kTileBytes);
+      for (int w = 0; w < 2; ++w)
+        for (int hf = 0; hf < 2; ++hf)
+          tma_load_4d(smem_base + kSmemQ + w * kTileBytes + hf * kHalfBytes, tmQ, &bars->q_full, hf * 64,
+                      u.q_tok + w * kTile, u.h, u.b);
+    }
+    ++n_units;
+    for (int it = 0; it < 2 * u.T; ++it, ++item) {   // 2*jt = K tile jt, 2*jt+1 = V tile jt
+      const uint32_t slot = item % kSlots, use = item / kSlots;
+      if (use > 0 && !mbar_wait(&bars->kv_empty[slot], (use - 1) & 1, bars, a.st, 30)) return;
+      if (lane == 0) {
+        const int jt = it >> 1;
+        const bool is_v = it & 1;
+        const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
+        unsigned long long* bar = &bars->kv_full[slot];
+        mbar_expect_tx(bar, kTileBytes);
+        if (jt < u.n_past_tiles) {
+          const CUtensorMap* tm = is_v ? tmVb : tmKb;
+          for (int q = 0; q < bpt; ++q) {
+            const int li = jt * bpt + q;
+            // boxes beyond the list read past the end of the tensor and arrive as zeros
+            const int tok = li < u.n_past ? u.list[li] * a.blk : a.n;
+            for (int hf = 0; hf < 2; ++hf)
+              tma_load_4d(dst + hf * kHalfBytes + q * a.blk * 128, tm, bar, hf * 64, tok, u.kvh, u.b);
+          }
+        } else {
+          const CUtensorMap* tm = is_v ? tmVt : tmKt;
+          const int ci = jt - u.n_past_tiles;
+          const int tok = ci < u.n_cont ? u.c_tok + ci * kTile : u.d_tok + (ci - u.n_cont) * kTile;
+          for (int hf = 0; hf < 2; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, bar, hf * 64, tok, u.kvh, u.b);
+        }
+      }
+      __syncwarp();
+    }
   }
 }
 
@@ -443,87 +513,65 @@ __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint3
     umma_ts(d_tmem, p_tmem + kk * 8, desc_at(base, v_smem + kk * 16 * 128), kIdescPV, (acc || kk > 0) ? 1u : 0u);
 }
 
-__device__ __forceinline__ void mma_role(const Args& a, const Unit& u, Bars* bars, uint32_t smem_base, int lane) {
+__device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t smem_base, int lane) {
   const uint32_t tm = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
   const uint32_t tS[2] = {tm, tm + 128}, tO[2] = {tm + 256, tm + 384};
   const uint32_t qA = smem_base + kSmemQ, qB = qA + kTileBytes;
-  const int T = u.T, TA = u.T - 1;
-  auto slot_addr = [&](int item) { return smem_base + kSmemKV + (item % kSlots) * kTileBytes; };
-  auto full_wait = [&](int item) {
+  uint32_t item0 = 0;                 // first K/V item of the current unit
+  uint32_t nA = 0, nB = 0;            // P tiles consumed so far per query tile (all units)
+  uint32_t n_units = 0;
+  auto slot_addr = [&](uint32_t item) { return smem_base + kSmemKV + (item % kSlots) * kTileBytes; };
+  auto full_wait = [&](uint32_t item) {
     return mbar_wait(&bars->kv_full[item % kSlots], (item / kSlots) & 1, bars, a.st, 40);
   };
-  if (!mbar_wait(&bars->q_full, 0, bars, a.st, 41)) return;
-  if (!full_wait(0)) return;
-  tc_fence_after();
-#ifdef CP_TRACE
-  if (blockIdx.x == 0) {
-    // MMA throughput probes: 64 back-to-back instructions of each kind into scratch accumulators
-    long long* tb = reinterpret_cast<long long*>(reinterpret_cast<char*>(a.st) + 256) + 3000;
-    for (int kind = 0; kind < 4; ++kind) {
-      const long long t0 = clock64();
-      {
-        for (int rep = 0; rep < 8; ++rep) {
-          if (kind == 0) issue_qk(tS[0], qA, slot_addr(0));                 // SS, N=128
-          else if (kind == 1) issue_pv(tO[0], tS[1], slot_addr(0), true);   // TS, N=128
-          else if (kind == 2) {                                             // SS, N=64
-            const uint64_t base = desc_base(16);
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-              umma_ss(tS[0], desc_at(base, qA + off), desc_at(base, slot_addr(0) + off), idesc, 1);
-            }
-          } else {                                                          // SS, N=256 (rows run on into the next buffer)
-            const uint64_t base = desc_base(16);
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
-            for (int kk = 0; kk < 8; ++kk) {
-              const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-              umma_ss(tS[0], desc_at(base, qA + off), desc_at(base, qA + off), idesc, 1);
-            }
-          }
-        }
-        umma_commit(&bars->dbg);
+  for (uint32_t q = 0;; ++q) {
+    bool got;
+    const int x = receive_unit(a, bars, q, lane, &got);
+    if (!got || x >= a.n_units || stop_requested(a, bars)) return;
+    const Unit u = decode_unit(a, x);
+    if (!unit_ok(a, u, lane)) continue;
+    const int T = u.T, TA = u.T - 1;
+    if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;
+    if (!full_wait(item0)) return;
+    tc_fence_after();
+    issue_qk(tS[0], qA, slot_addr(item0)); umma_commit(&bars->s_full[0]);
+    issue_qk(tS[1], qB, slot_addr(item0)); umma_commit(&bars->s_full[1]);
+    umma_commit(&bars->kv_empty[item0 % kSlots]);
+    for (int jt = 0; jt < T; ++jt) {
+      const bool has_next = jt + 1 < T;
+      const uint32_t iv = item0 + 2 * jt + 1, ik = item0 + 2 * (jt + 1);
+      if (has_next && !full_wait(ik)) return;
+      if (!full_wait(iv)) return;
+      const uint32_t v_smem = slot_addr(iv), kn_smem = slot_addr(ik);
+      const bool tr = blockIdx.x == 0 && q == 0 && lane == 0 && jt < 64;
+      CP_STAMP(tr, 2048 + jt * 8 + 0);
+      if (jt < TA) {
+        if (!mbar_wait(&bars->p_full[0], nA & 1, bars, a.st, 42)) return;
+        ++nA;
+        CP_STAMP(tr, 2048 + jt * 8 + 1);
+        tc_fence_after();
+        issue_pv(tO[0], tS[0], v_smem, jt > 0);
+        if (jt + 1 < TA) { issue_qk(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
+        else umma_commit(&bars->o_done[0]);
       }
-      __syncwarp();
-      const long long t1 = clock64();
-      mbar_wait(&bars->dbg, kind & 1, bars, a.st, 99);
-      const long long t2 = clock64();
-      if (lane == 0) { tb[kind * 2] = t1 - t0; tb[kind * 2 + 1] = t2 - t0; }
-    }
-    tc_fence_after();
-  }
-#endif
-  issue_qk(tS[0], qA, slot_addr(0)); umma_commit(&bars->s_full[0]);
-  issue_qk(tS[1], qB, slot_addr(0)); umma_commit(&bars->s_full[1]);
-  umma_commit(&bars->kv_empty[0]);
-  for (int jt = 0; jt < T; ++jt) {
-    const bool has_next = jt + 1 < T;
-    if (has_next && !full_wait(2 * (jt + 1))) return;
-    if (!full_wait(2 * jt + 1)) return;
-    const uint32_t v_smem = slot_addr(2 * jt + 1);
-    const uint32_t kn_smem = slot_addr(2 * (jt + 1));
-    const bool tr = blockIdx.x == 0 && lane == 0 && jt < 64;
-    CP_STAMP(tr, 2048 + jt * 8 + 0);
-    if (jt < TA) {
-      if (!mbar_wait(&bars->p_full[0], jt & 1, bars, a.st, 42)) return;
-      CP_STAMP(tr, 2048 + jt * 8 + 1);
+      CP_STAMP(tr, 2048 + jt * 8 + 2);
+      if (!mbar_wait(&bars->p_full[1], nB & 1, bars, a.st, 43)) return;
+      ++nB;
+      CP_STAMP(tr, 2048 + jt * 8 + 3);
       tc_fence_after();
-      issue_pv(tO[0], tS[0], v_smem, jt > 0);
-      if (jt + 1 < TA) { issue_qk(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
-      else umma_commit(&bars->o_done[0]);
+      issue_pv(tO[1], tS[1], v_smem, jt > 0);
+      umma_commit(&bars->kv_empty[iv % kSlots]);
+      if (has_next) {
+        issue_qk(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
+        umma_commit(&bars->kv_empty[ik % kSlots]);
+        if (jt + 1 == T - 1) umma_commit(&bars->q_empty);   // that was the unit's last QK^T: Q may be replaced
+      } else {
+        umma_commit(&bars->o_done[1]);
+      }
+      CP_STAMP(tr, 2048 + jt * 8 + 4);
     }
-    CP_STAMP(tr, 2048 + jt * 8 + 2);
-    if (!mbar_wait(&bars->p_full[1], jt & 1, bars, a.st, 43)) return;
-    CP_STAMP(tr, 2048 + jt * 8 + 3);
-    tc_fence_after();
-    issue_pv(tO[1], tS[1], v_smem, jt > 0);
-    umma_commit(&bars->kv_empty[(2 * jt + 1) % kSlots]);
-    if (has_next) {
-      issue_qk(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
-      umma_commit(&bars->kv_empty[(2 * (jt + 1)) % kSlots]);
-    } else {
-      umma_commit(&bars->o_done[1]);
-    }
-    CP_STAMP(tr, 2048 + jt * 8 + 4);
+    item0 += 2 * T;
+    ++n_units;
   }
 }
 
@@ -540,11 +588,10 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
   if (threadIdx.x == 0) {
     mbar_init(&bars->q_full, 1);
+    mbar_init(&bars->q_empty, 1);
     for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->kv_full[i], 1); mbar_init(&bars->kv_empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->s_full[i], 1); mbar_init(&bars->p_full[i], 128); mbar_init(&bars->o_done[i], 1); }
-#ifdef CP_TRACE
-    mbar_init(&bars->dbg, 1);
-#endif
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->sched_full[i], 1); mbar_init(&bars->sched_empty[i], 9); }
     bars->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -557,37 +604,16 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   __syncthreads();
   tc_fence_after();
 
-  Unit u = decode_unit(a);
-  // once any CTA has reported a timeout the remaining CTAs do no work (keeps a broken run short)
-  if (a.st != nullptr && *reinterpret_cast<volatile int32_t*>(&a.st->code) == CP_ERR_TIMEOUT) u.ok = false;
-  // the list contract: ascending past blocks, then exactly the r diagonal blocks
-  if (!a.dense) {
-    bool ok = u.ok;
-    if (ok) {
-      const int c = u.n_past + a.r;
-      for (int i = threadIdx.x; i < c; i += kThreads) {
-        const int v = u.list[i];
-        if (i >= u.n_past) ok = ok && (v == u.seg_j * a.r + (i - u.n_past));
-        else ok = ok && v >= 0 && v < u.seg_j * a.r && (i == 0 || u.list[i - 1] < v);
-      }
-    }
-    ok = __syncthreads_and(ok);
-    if (!ok && threadIdx.x == 0) report(a.st, CP_ERR_BOUNDS, 1, u.b, u.h, u.seg_j, u.n_past + a.r);
-    u.ok = ok;
-  }
-
   // Register re-partition.  The pool is what the CTA was launched with (384 threads x 168):
-  // 256 x 224 + 128 x 56 = 64512 fits it exactly; asking for more would block forever.
-  static_assert(256 * 224 + 128 * 56 <= kThreads * 168, "setmaxnreg budget exceeds the launch allocation");
+  // 256 x 216 + 128 x 64 = 63488 fits; asking for more than the pool would block forever.
+  static_assert(256 * 216 + 128 * 64 <= kThreads * 168, "setmaxnreg budget exceeds the launch allocation");
   if (warp < 8) {
-    reg_inc<224>();
-    if (u.ok) softmax_role(a, u, bars, warp >> 2, warp & 3, lane);
+    reg_inc<216>();
+    softmax_role(a, bars, warp >> 2, warp & 3, lane);
   } else {
-    reg_dec<56>();
-    if (u.ok) {
-      if (warp == 8) producer_role(a, u, bars, smem_base, &tmQ, &tmKb, &tmVb, &tmKt, &tmVt, lane);
-      else if (warp == 9) mma_role(a, u, bars, smem_base, lane);
-    }
+    reg_dec<64>();
+    if (warp == 8) producer_role(a, bars, smem_base, &tmQ, &tmKb, &tmVb, &tmKt, &tmVt, lane);
+    else if (warp == 9) mma_role(a, bars, smem_base, lane);
   }
   if (bars->abort_flag) {
     // give copies and MMAs still in flight time to land before the CTA's resources go away
@@ -654,7 +680,15 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
   if (cudaFuncSetAttribute(attention_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)
     return CP_ERR_CUDA;
-  attention_sm100_kernel<<<unsigned(units), kThreads, kSmemTotal, s>>>(tmQ, tmKb, tmVb, tmKt, tmVt, a);
+  a.n_units = int(units);
+  a.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(st) + 128);   // inside the status block
+  if (cudaMemsetAsync(a.work_counter, 0, sizeof(unsigned int), s) != cudaSuccess) return CP_ERR_CUDA;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return CP_ERR_CUDA;
+  // persistent CTAs, one per SM (the kernel takes all of an SM's tensor memory and shared memory)
+  const unsigned grid = unsigned(units < sms ? units : sms);
+  attention_sm100_kernel<<<grid, kThreads, kSmemTotal, s>>>(tmQ, tmKb, tmVb, tmKt, tmVt, a);
   return check_launch();
 }
 
