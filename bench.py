@@ -162,7 +162,7 @@ def run_reference(args, cfg):
     import oracle.build
     oracle.build.build()
     Q, K, V = make_qkv(cfg)
-    n_rows = 256
+    n_rows = min(cfg.seq_len, 8192)
     cores = os.cpu_count()
     for i in range(args.warmup):
         oracle_step(cfg, Q, K, V, i % cfg.n_q_heads, n_rows, i)

@@ -55,7 +55,10 @@ typedef enum { CP_BF16 = 0, CP_F32 = 1 } cp_dtype;
 
 enum {
   CP_FLAG_MASK_BEFORE_SOFTMAX = 1, /* estimate: normalise each score map over visible blocks only */
-  CP_FLAG_FORCE_SIMT = 2           /* attention: use the SIMT kernel even where tensor cores apply */
+  CP_FLAG_FORCE_SIMT = 2,          /* attention: use the SIMT kernel even where tensor cores apply */
+  CP_FLAG_TEST_WITHHOLD_V = 4      /* test hook for the bounded waits of the tensor-core kernel: V tiles are
+                                      never loaded, so a pipeline wait expires after about 2 s, the kernel
+                                      drains and the status block reads CP_ERR_TIMEOUT (outputs invalid) */
 };
 
 typedef struct {

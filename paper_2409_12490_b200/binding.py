@@ -20,6 +20,7 @@ CP_OK = 0
 CP_BF16, CP_F32 = 0, 1
 FLAG_MASK_BEFORE_SOFTMAX = 1
 FLAG_FORCE_SIMT = 2
+FLAG_TEST_WITHHOLD_V = 4
 
 EXPORTS = (
     "critiprefill_workspace_bytes", "critiprefill_estimate", "critiprefill_select",

@@ -60,6 +60,7 @@ struct Args {
   float sm_scale;
   int dense;
   int n_units;
+  int withhold_v;               // test hook: the producer never issues V tiles, so a bounded wait must expire
   unsigned int* work_counter;   // next unit to hand out (zeroed by the host before the launch)
 };
 
@@ -470,7 +471,7 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
     for (int it = 0; it < 2 * u.T; ++it, ++item) {   // 2*jt = K tile jt, 2*jt+1 = V tile jt
       const uint32_t slot = item % kSlots, use = item / kSlots;
       if (use > 0 && !mbar_wait(&bars->kv_empty[slot], (use - 1) & 1, bars, a.st, 30)) return;
-      if (lane == 0) {
+      if (lane == 0 && !(a.withhold_v && (it & 1))) {
         const int jt = it >> 1;
         const bool is_v = it & 1;
         const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
@@ -681,6 +682,7 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
   if (cudaFuncSetAttribute(attention_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)
     return CP_ERR_CUDA;
   a.n_units = int(units);
+  a.withhold_v = (p.flags & CP_FLAG_TEST_WITHHOLD_V) ? 1 : 0;
   a.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(st) + 128);   // inside the status block
   if (cudaMemsetAsync(a.work_counter, 0, sizeof(unsigned int), s) != cudaSuccess) return CP_ERR_CUDA;
   int dev = 0, sms = 0;

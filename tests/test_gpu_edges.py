@@ -1,0 +1,102 @@
+"""Edge cases of the CUDA path against the oracle: smallest shapes, budgets that hold only the
+diagonal, large logits (rescale path), the SIMT fallback shapes, and the bounded-wait status."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2409_12490_b200 import CONFIGS
+from paper_2409_12490_b200 import binding as cp
+from paper_2409_12490_b200.inputs import make_qkv, make_uniform_qkv
+
+from helpers import TOL_BF16_MAX, TOL_BF16_MEAN, assert_attention_close, attention_errors, compare_scores, compare_selection, f32, oracle_scores, problem, to_dev
+
+pytestmark = pytest.mark.gpu
+
+BASE = CONFIGS["C2"].with_(name="edge", seq_len=1024, n_q_heads=2, n_kv_heads=1, segment_size=256,
+                           block_size=128, budget_tokens=256, n_clusters=8)
+
+
+def full_path_vs_oracle(cfg, Q, K, V, flags=0, tol=(TOL_BF16_MAX, TOL_BF16_MEAN)):
+    prob = problem(cfg, flags=flags)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    O, S, idx, cnt = cp.prefill_layer(prob, Qd, Kd, Vd, ws)
+    assert cp.device_status(ws) == 0
+    S_ref = oracle_scores(cfg, Q, K)
+    compare_scores(S, S_ref)
+    idx_ref, cnt_ref = oracle.select(S_ref, cfg.segment_size, cfg.block_size, cfg.budget_blocks)
+    assert compare_selection(idx, cnt, idx_ref, cnt_ref, S_ref, cfg.r)[1] == 0
+    O_ref, _ = oracle.sparse_attention(Q, K, V, idx.cpu().numpy(), cnt.cpu().numpy(), cfg.segment_size, cfg.block_size,
+                                       f32(1.0 / np.sqrt(cfg.head_dim)))
+    assert_attention_close(O, O_ref, *tol)
+    return O
+
+
+def test_budget_holds_only_the_diagonal_blocks():
+    cfg = BASE                                   # k = r = 2: no past block is ever taken
+    full_path_vs_oracle(cfg, *make_qkv(cfg))
+
+
+def test_single_unit_sequence():
+    cfg = BASE.with_(seq_len=256)                # one segment, one 256-row unit, two tiles
+    full_path_vs_oracle(cfg, *make_qkv(cfg))
+
+
+def test_many_small_units_batch3():
+    cfg = BASE.with_(batch=3, n_q_heads=4, n_kv_heads=4, seq_len=2048, block_size=32, budget_tokens=352)
+    full_path_vs_oracle(cfg, *make_qkv(cfg))     # 11 blocks of 32: ragged last gathered tile
+
+
+def test_large_logits_exercise_the_rescale_path():
+    cfg = BASE.with_(seq_len=2048, budget_tokens=1024)
+    Q, K, V = make_uniform_qkv(1, 2, 1, 2048, 128, seed=11, scale=1.0)
+    Q = (Q.float() * 6.0).to(torch.bfloat16)     # logits up to ~ +-60: row maxima jump between tiles
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    Od = cp.dense_attention(prob, Qd, Kd, Vd, ws)
+    assert cp.device_status(ws) == 0
+    O_ref, _ = oracle.dense_attention(Q, K, V, f32(1.0 / np.sqrt(128)))
+    # Peaked rows put almost all weight on a few keys, so the unit-scale tolerance does not apply.
+    # From the arithmetic: each probability is rounded to bf16 (unit roundoff 2^-8) while the row sum
+    # is taken before rounding, and O is rounded to bf16 once more, so
+    #   |O_gpu - O| <= 2^-8 * (sum_u p_u |v_u| + |O|) <= 2^-7 * max|V|.
+    bound = 2.0 ** -7 * float(V.float().abs().max())
+    mx, mean = attention_errors(Od, O_ref)
+    assert mx <= bound and mean <= TOL_BF16_MEAN, (mx, mean, bound)
+
+
+@pytest.mark.parametrize("seg,blk,d", [(128, 32, 128), (384, 64, 128), (256, 64, 64)])
+def test_shapes_served_by_the_simt_kernel(seg, blk, d):
+    cfg = BASE.with_(seq_len=768, segment_size=seg, block_size=blk, budget_tokens=max(seg, 256), head_dim=d)
+    full_path_vs_oracle(cfg, *make_qkv(cfg))
+
+
+def test_fp32_path_with_strided_output():
+    cfg = CONFIGS["C1"].with_(seq_len=512)
+    Q, K, V = make_qkv(cfg)
+    O = full_path_vs_oracle(cfg, Q, K, V, tol=(1e-5, 1e-6))
+    assert O.dtype == torch.float32
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """Failure detection without a fault: with the V loads withheld a pipeline wait runs out, the
+    kernel drains, the status reads CP_ERR_TIMEOUT, and the next call on the same context works."""
+    cfg = BASE.with_(seq_len=256)
+    Q, K, V = make_qkv(cfg)
+    S_ref = oracle_scores(cfg, Q, K)
+    idx_ref, cnt_ref = oracle.select(S_ref, cfg.segment_size, cfg.block_size, cfg.budget_blocks)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    idx, cnt = torch.from_numpy(idx_ref).cuda(), torch.from_numpy(cnt_ref).cuda()
+    prob = problem(cfg, flags=cp.FLAG_TEST_WITHHOLD_V)
+    ws = cp.alloc_workspace(prob)
+    cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws)
+    assert cp.device_status(ws) == 6
+    ws.zero_()
+    prob = problem(cfg)
+    O = cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws)
+    assert cp.device_status(ws) == 0
+    O_ref, _ = oracle.sparse_attention(Q, K, V, idx_ref, cnt_ref, cfg.segment_size, cfg.block_size,
+                                       f32(1.0 / np.sqrt(cfg.head_dim)))
+    assert_attention_close(O, O_ref)

@@ -8,7 +8,7 @@ from paper_2409_12490_b200 import CONFIGS
 from paper_2409_12490_b200 import binding as cp
 from paper_2409_12490_b200.inputs import make_qkv, make_uniform_qkv
 
-from helpers import (TOL_BF16_MAX, TOL_BF16_MEAN, TOL_F32, attention_errors, compare_scores, compare_selection,
+from helpers import (TOL_BF16_MAX, TOL_BF16_MEAN, TOL_F32, assert_attention_close, attention_errors, compare_scores, compare_selection,
                      f32, oracle_scores, problem, to_dev)
 
 pytestmark = pytest.mark.gpu
@@ -97,8 +97,7 @@ def test_attention_bf16_matches_oracle(blk, budget, flags):
     cfg = SMALL_BF16.with_(block_size=blk, budget_tokens=budget)
     Q, K, V = make_qkv(cfg)
     O, lse, O_ref, lse_ref = _sparse_case(cfg, Q, K, V, flags)
-    mx, mean = attention_errors(O, O_ref)
-    assert mx <= TOL_BF16_MAX and mean <= TOL_BF16_MEAN, (mx, mean)
+    assert_attention_close(O, O_ref)
     assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 2e-3
 
 
@@ -112,8 +111,7 @@ def test_dense_bf16_matches_oracle_and_full_budget_sparse():
     assert cp.device_status(ws) == 0
     sm = f32(1.0 / np.sqrt(cfg.head_dim))
     O_ref, lse_ref = oracle.dense_attention(Q, K, V, sm)
-    mx, mean = attention_errors(O, O_ref)
-    assert mx <= TOL_BF16_MAX and mean <= TOL_BF16_MEAN, (mx, mean)
+    assert_attention_close(O, O_ref)
     assert np.abs(lse.cpu().numpy() - lse_ref).max() <= 2e-3
 
 
@@ -141,8 +139,7 @@ def test_uniform_inputs_batch2_strided():
     assert cp.device_status(ws) == 0
     O_ref, _ = oracle.sparse_attention(Q, K, V, idx_ref, cnt_ref, cfg.segment_size, cfg.block_size,
                                        f32(1.0 / np.sqrt(d)))
-    mx, mean = attention_errors(O, O_ref)
-    assert mx <= TOL_BF16_MAX and mean <= TOL_BF16_MEAN, (mx, mean)
+    assert_attention_close(O, O_ref)
 
 
 def test_select_with_ties_matches_oracle():
