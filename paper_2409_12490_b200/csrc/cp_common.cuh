@@ -9,7 +9,7 @@
 namespace cp {
 
 constexpr int kStatusBytes = 256;   // head of the workspace: status word + diagnostics
-constexpr int kMaxBlocksN2 = 6144;  // estimate keeps 4*n2 fp64 logits per head in shared memory
+constexpr int kMaxBlocksN2 = 8192;  // estimate: fp64 logits in the shared memory of up to 8 clustered CTAs; select: 32 keys/thread
 
 // Derived sizes of one problem.
 struct Dims {

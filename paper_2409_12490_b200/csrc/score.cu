@@ -5,6 +5,7 @@
 //   ln S = max( ln((S1+S3)/2), ln((S2+S4)/2) ),  mask,  ln(alpha S + (1-alpha) S').
 // The representatives are exact in the input dtype, every product is exact in fp64, so this
 // differs from an fp64 CPU evaluation only by summation order and libm rounding.
+#include <cooperative_groups.h>
 #include <math_constants.h>
 
 #include "cp_common.cuh"
@@ -28,20 +29,28 @@ __device__ __forceinline__ double logaddexp(double a, double b) {
   return hi + log1p(exp(d));
 }
 
-// Shared memory: logits lg[U][4][n2].
+// Shared memory: logits lg[U][4][nb] for the nb key blocks this CTA owns.  When the 4*U*n2 logits
+// of a row group do not fit one CTA's shared memory, CL CTAs of a thread-block cluster split the
+// key blocks and merge their per-row (max, sum) pairs through distributed shared memory.
 template <typename T, int D, int U>
 __global__ void __launch_bounds__(kThreads)
 score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __restrict__ Kmax,
              const T* __restrict__ Kmin, const double* __restrict__ S_prev, double* __restrict__ S_out,
              int Hq, int g, int n1, int n2, int seg, int blk, double est_scale, double ln_alpha,
-             double ln_1m_alpha, int fuse, int mask_first) {
+             double ln_1m_alpha, int fuse, int mask_first, int CL, int nb) {
   extern __shared__ double smem[];
-  double* lg = smem;                                // [U][4][n2]
+  double* lg = smem;                                // [U][4][nb]
   __shared__ double stat[4 * U];
+  __shared__ double2 part[4 * U];                   // this CTA's (max, sum exp) per logit row
+
+  // cluster rank -> owned key blocks [b_lo, b_lo + nloc)
+  const int rank = CL > 1 ? int(blockIdx.x % CL) : 0;
+  const int b_lo = rank * nb;
+  const int nloc = max(0, min(n2, b_lo + nb) - b_lo);
 
   // CTA -> (b, kv head, head subgroup, segment)
   const int groups = g / U;
-  int x = blockIdx.x;
+  int x = blockIdx.x / CL;
   const int j = x % n1; x /= n1;
   const int sub = x % groups; x /= groups;
   const int kvh = x;                                 // b*Hkv + kv head
@@ -72,9 +81,9 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
 #pragma unroll
     for (int ks = 0; ks < KS; ++ks) afrag[ks] = u < U ? to_f64(src[ks]) : 0.0;
   }
-  const int n_tiles = (n2 + 7) / 8;
+  const int n_tiles = (nloc + 7) / 8;
   for (int t = warp; t < n_tiles; t += kWarps) {
-    const int bblk = min(t * 8 + grp, n2 - 1);          // this lane's B column (clamped in a ragged last tile)
+    const int bblk = b_lo + min(t * 8 + grp, nloc - 1);  // this lane's B column (clamped in a ragged last tile)
     const uint4* pmx = reinterpret_cast<const uint4*>(kmx_base + size_t(bblk) * D + quad * KS);
     const uint4* pmn = reinterpret_cast<const uint4*>(kmn_base + size_t(bblk) * D + quad * KS);
     uint4 vx[NV], vn[NV];
@@ -100,11 +109,11 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
     if (u < U) {
 #pragma unroll
       for (int i = 0; i < 2; ++i) {
-        const int bb = t * 8 + quad * 2 + i;
-        if (bb < n2) {
-          const bool hide = mask_first && bb >= visible;
-          lg[(u * 4 + rep * 2 + 0) * n2 + bb] = hide ? -CUDART_INF : (i ? cx1 : cx0) * est_scale;
-          lg[(u * 4 + rep * 2 + 1) * n2 + bb] = hide ? -CUDART_INF : (i ? cn1 : cn0) * est_scale;
+        const int lb = t * 8 + quad * 2 + i;           // local block index
+        if (lb < nloc) {
+          const bool hide = mask_first && b_lo + lb >= visible;
+          lg[(u * 4 + rep * 2 + 0) * nb + lb] = hide ? -CUDART_INF : (i ? cx1 : cx0) * est_scale;
+          lg[(u * 4 + rep * 2 + 1) * nb + lb] = hide ? -CUDART_INF : (i ? cn1 : cn0) * est_scale;
         }
       }
     }
@@ -115,35 +124,54 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   // row, so only shuffles are needed; terms more than e^-50 below the maximum are skipped
 #pragma unroll 1
   for (int rI = warp; rI < 4 * U; rI += kWarps) {
-    const double* rowp = lg + rI * n2;
+    const double* rowp = lg + rI * nb;
     double m = -CUDART_INF;
-    for (int bb = lane; bb < n2; bb += 32) m = fmax(m, rowp[bb]);
+    for (int lb = lane; lb < nloc; lb += 32) m = fmax(m, rowp[lb]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
     double sum = 0.0;
 #pragma unroll 4
-    for (int bb = lane; bb < n2; bb += 32) {
-      const double d = rowp[bb] - m;
+    for (int lb = lane; lb < nloc; lb += 32) {
+      const double d = rowp[lb] - m;
       if (d > -50.0) sum += exp(d);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) stat[rI] = m + log(sum);
+    if (lane == 0) part[rI] = make_double2(m, sum);
+  }
+  __syncthreads();
+  if (CL > 1) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    cluster.sync();                                   // every CTA's partials are in place
+    if (tid < 4 * U) {
+      double M = -CUDART_INF;
+      for (int r = 0; r < CL; ++r) M = fmax(M, cluster.map_shared_rank(part, r)[tid].x);
+      double Ssum = 0.0;
+      for (int r = 0; r < CL; ++r) {
+        const double2 pr = cluster.map_shared_rank(part, r)[tid];
+        if (pr.y > 0.0) Ssum += pr.y * exp(pr.x - M);
+      }
+      stat[tid] = M + log(Ssum);
+    }
+    cluster.sync();                                   // nobody leaves while its partials may still be read
+  } else if (tid < 4 * U) {
+    stat[tid] = part[tid].x + log(part[tid].y);
   }
   __syncthreads();
 
-  // combine (lines 11-12), mask (13), fusion (14) over the U rows of this CTA, flattened
+  // combine (lines 11-12), mask (13), fusion (14) over this CTA's blocks of the U rows, flattened
   const double ln2 = 0.693147180559945309417232121458;
 #pragma unroll 2
-  for (int e = tid; e < U * n2; e += kThreads) {
-    const int u = e / n2, bb = e - u * n2;
+  for (int e = tid; e < U * nloc; e += kThreads) {
+    const int u = e / nloc, lb = e - u * nloc, bb = b_lo + lb;
     double v;
     if (bb >= visible) {
       v = -CUDART_INF;
     } else {
-      const double* l = lg + u * 4 * n2;
-      const double L1 = l[bb] - stat[u * 4 + 0], L2 = l[n2 + bb] - stat[u * 4 + 1];
-      const double L3 = l[2 * n2 + bb] - stat[u * 4 + 2], L4 = l[3 * n2 + bb] - stat[u * 4 + 3];
+      const double* l = lg + u * 4 * nb;
+      const double L1 = l[lb] - stat[u * 4 + 0], L2 = l[nb + lb] - stat[u * 4 + 1];
+      const double L3 = l[2 * nb + lb] - stat[u * 4 + 2], L4 = l[3 * nb + lb] - stat[u * 4 + 3];
       const double Lmax = logaddexp(L1, L3) - ln2;   // ln (S1+S3)/2
       const double Lmin = logaddexp(L2, L4) - ln2;   // ln (S2+S4)/2
       v = fmax(Lmax, Lmin);
@@ -155,29 +183,44 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
 
 template <typename T, int D, int U>
 int launch_u(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
-             double est_scale, double alpha, int fuse, int mask_first, cudaStream_t st) {
-  const size_t smem = sizeof(double) * (4 * size_t(U) * m.n2);
+             double est_scale, double alpha, int fuse, int mask_first, int CL, int nb, cudaStream_t st) {
+  const size_t smem = sizeof(double) * (4 * size_t(U) * nb);
   auto kern = score_kernel<T, D, U>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
     return CP_ERR_CUDA;
-  const long long ctas = (long long)m.B * m.Hkv * (m.g / U) * m.n1;
+  const long long ctas = (long long)m.B * m.Hkv * (m.g / U) * m.n1 * CL;
   if (ctas > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
-  kern<<<unsigned(ctas), kThreads, smem, st>>>(
-      reinterpret_cast<const T*>(ws + w.qmax), reinterpret_cast<const T*>(ws + w.qmin),
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(ctas));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = unsigned(CL); attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = CL > 1 ? 1 : 0;
+  const cudaError_t e = cudaLaunchKernelEx(
+      &cfg, kern, reinterpret_cast<const T*>(ws + w.qmax), reinterpret_cast<const T*>(ws + w.qmin),
       reinterpret_cast<const T*>(ws + w.kmax), reinterpret_cast<const T*>(ws + w.kmin), S_prev, S_out,
-      m.Hq, m.g, m.n1, m.n2, m.seg, m.blk, est_scale, log(alpha), log1p(-alpha), fuse, mask_first);
-  return check_launch();
+      m.Hq, m.g, m.n1, m.n2, m.seg, m.blk, est_scale, log(alpha), log1p(-alpha), fuse, mask_first, CL, nb);
+  return e == cudaSuccess ? check_launch() : CP_ERR_CUDA;
 }
 
 template <typename T, int D>
 int launch_t(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
              double est_scale, double alpha, int fuse, int mask_first, cudaStream_t st) {
-  // as many heads per CTA as divide the group and keep the logits within ~200 KB of shared memory
+  // as many heads per CTA as divide the group (the fp64 MMA has 8 rows = 4 heads x 2 representatives);
+  // key blocks are split over a cluster of 1, 2, 4 or 8 CTAs until the logits fit ~200 KB per CTA
   const size_t budget = 200 * 1024;
-  auto fits = [&](int U) { return m.g % U == 0 && sizeof(double) * (4 * size_t(U) * m.n2) <= budget; };
-  if (fits(4)) return launch_u<T, D, 4>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, st);
-  if (fits(2)) return launch_u<T, D, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, st);
-  if (fits(1)) return launch_u<T, D, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, st);
+  const int U = m.g % 4 == 0 ? 4 : (m.g % 2 == 0 ? 2 : 1);
+  for (int CL = 1; CL <= 8; CL *= 2) {
+    const int nb = (((m.n2 + CL - 1) / CL) + 7) & ~7;
+    if (sizeof(double) * 4 * size_t(U) * nb > budget) continue;
+    if (U == 4) return launch_u<T, D, 4>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
+    if (U == 2) return launch_u<T, D, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
+    return launch_u<T, D, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
+  }
   return CP_ERR_UNSUPPORTED;
 }
 

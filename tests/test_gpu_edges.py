@@ -100,3 +100,25 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     O_ref, _ = oracle.sparse_attention(Q, K, V, idx_ref, cnt_ref, cfg.segment_size, cfg.block_size,
                                        f32(1.0 / np.sqrt(cfg.head_dim)))
     assert_attention_close(O, O_ref)
+
+
+@pytest.mark.parametrize("n,seg,blk", [(8192, 64, 4), (16384, 128, 4), (8224, 8, 4)])
+def test_many_key_blocks_split_over_a_cluster(n, seg, blk):
+    """n2 = 2048 / 4096 / 2056 key blocks: the score kernel spreads them over 2 or 4 clustered CTAs
+    (the last case with a ragged split); estimate and select must still match the oracle."""
+    cfg = CONFIGS["C1"].with_(name="wide", seq_len=n, n_q_heads=4, n_kv_heads=1, head_dim=64, segment_size=seg,
+                              block_size=blk, budget_tokens=max(2 * seg, 64 * blk), n_clusters=8)
+    Q, K, _ = make_qkv(cfg)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd = to_dev(Q, K)
+    S = cp.estimate(prob, Qd, Kd, ws)
+    idx, cnt = cp.select(prob, S, ws)
+    S_ref = oracle_scores(cfg, Q, K)
+    compare_scores(S, S_ref)
+    idx_ref, cnt_ref = oracle.select(S_ref, cfg.segment_size, cfg.block_size, cfg.budget_blocks)
+    assert compare_selection(idx, cnt, idx_ref, cnt_ref, S_ref, cfg.r)[1] == 0
+    # a fused second layer through the same path
+    Q1, K1, _ = make_qkv(cfg, layer=1)
+    S1 = cp.estimate(prob, *to_dev(Q1, K1), ws, S_prev=S)
+    compare_scores(S1, oracle_scores(cfg, Q1, K1, S_prev=S_ref))
