@@ -122,3 +122,20 @@ def test_many_key_blocks_split_over_a_cluster(n, seg, blk):
     Q1, K1, _ = make_qkv(cfg, layer=1)
     S1 = cp.estimate(prob, *to_dev(Q1, K1), ws, S_prev=S)
     compare_scores(S1, oracle_scores(cfg, Q1, K1, S_prev=S_ref))
+
+
+def test_host_pipelined_layer_equals_resident_path():
+    from paper_2409_12490_b200.pipeline import HostPipelinedLayer
+    cfg = CONFIGS["C2"].with_(name="pipe", seq_len=2048, n_q_heads=8, n_kv_heads=4, segment_size=256, block_size=64,
+                              budget_tokens=512, n_clusters=16)
+    Q, K, V = make_qkv(cfg)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    O_res, _, _, _ = cp.prefill_layer(prob, *to_dev(Q, K, V), ws)
+    hQ, hK, hV = Q.pin_memory(), K.pin_memory(), V.pin_memory()
+    hO = torch.empty_like(hQ).pin_memory()
+    layer = HostPipelinedLayer(prob)
+    layer(hQ, hK, hV, hO)
+    torch.cuda.synchronize()
+    assert layer.status() == 0 and cp.device_status(ws) == 0
+    assert torch.equal(hO, O_res.cpu())
