@@ -29,9 +29,10 @@ from paper_2409_12490_b200.inputs import make_qkv  # noqa: E402
 from paper_2409_12490_b200.sharding import RankInfo, aggregate_time_metric, layer_seed_for_rank, max_over_ranks  # noqa: E402
 
 METRIC = "128K prefill-attention ms (estimate+select+sparse attention, one layer)"
-# DRAM bytes per launch of the sparse attention kernel at the bench workload, from the ncu
-# capture summarised under profiles/ (None until one exists for the current kernel).
-ATTN_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) per launch of the sparse attention kernel, from the ncu captures
+# summarised in profiles/attention_sm100_kernel_C4_dram.md (C4, full size) and
+# profiles/attention_sm100_kernel_C3.md; None for workloads without a capture.
+ATTN_TRAFFIC_BYTES = {"C4": 2.80e9, "C3": 0.635e9}
 
 
 def load_peaks():
@@ -362,7 +363,8 @@ def run_ours(args, cfg):
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_tflops"], "peak_source": f"{peaks['source']} (burst)",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
-                "flops_per_launch": fl["executed"], "traffic": ATTN_TRAFFIC_BYTES}
+                "flops_per_launch": fl["executed"], "traffic": ATTN_TRAFFIC_BYTES.get(cfg.name),
+                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, ncu)"}
     summary_bytes = (dQ.numel() + dK.numel()) * dQ.element_size()
     out = {
         "metric": METRIC, "value": ms_per_step, "unit": "ms", "n_gpus": world, "steps": args.steps,
