@@ -97,3 +97,34 @@ def test_properties_at_full_size(c4):
     g = cfg.n_q_heads // cfg.n_kv_heads
     v0 = c4["V"][0, :, 0].repeat_interleave(g, dim=0)
     assert torch.equal(c4["O"][0, :, 0].cpu(), v0)
+
+
+def test_yi_shape_two_layer_chain_at_full_size():
+    """C5's shape (32 query / 4 KV heads, 128K tokens) with the score carried from layer 0 into layer 1
+    (Algorithm 1, line 14): scores and selection of one KV group against the oracle for both layers, and
+    layer 1's attention on sampled rows of that group."""
+    cfg = CONFIGS["C5"]
+    g = cfg.n_q_heads // cfg.n_kv_heads
+    prob = cp.Problem.from_config(cfg)
+    ws = cp.alloc_workspace(prob)
+    kvh = 2
+    hs = slice(kvh * g, (kvh + 1) * g)
+    S_prev_gpu, S_prev_ref = None, None
+    for layer in (0, 1):
+        Q, K, V = make_qkv(cfg, layer=layer)
+        Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+        S = cp.estimate(prob, Qd, Kd, ws, S_prev=S_prev_gpu)
+        idx, cnt = cp.select(prob, S, ws)
+        S_ref = oracle.estimate(Q[:, hs], K[:, kvh:kvh + 1], cfg.segment_size, cfg.block_size,
+                                est_scale=f32(cfg.est_scale), alpha=f32(cfg.alpha), S_prev=S_prev_ref)
+        compare_scores(S[:, hs], S_ref, atol=1e-9)
+        idx_ref, cnt_ref = oracle.select(S_ref, cfg.segment_size, cfg.block_size, cfg.budget_blocks)
+        assert compare_selection(idx[:, hs], cnt[:, hs], idx_ref, cnt_ref, S_ref, cfg.r)[1] == 0
+        S_prev_gpu, S_prev_ref = S, S_ref
+    O = cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws)
+    assert cp.device_status(ws) == 0
+    rng = np.random.default_rng(3)
+    rows = np.array([(0, kvh * g + int(rng.integers(g)), int(t)) for t in rng.integers(0, cfg.seq_len, 512)], dtype=np.int64)
+    O_ref, _ = oracle.sparse_attention_rows(Q, K, V, idx.cpu().numpy(), cnt.cpu().numpy(), cfg.segment_size,
+                                            cfg.block_size, f32(1.0 / np.sqrt(cfg.head_dim)), rows)
+    assert_attention_close(O[rows[:, 0], rows[:, 1], rows[:, 2]], O_ref)
