@@ -19,14 +19,14 @@
  *   - Tensor layout: Q and O are [batch, n_q_heads, seq_len, head_dim], K and V are
  *     [batch, n_kv_heads, seq_len, head_dim]; the three outer strides are given in ELEMENTS
  *     in cp_params, head_dim is contiguous.  Base pointers must be 16-byte aligned and the
- *     strides multiples of 8 elements (bf16) / 4 elements (fp32).
+ *     strides multiples of 8 elements (bf16, fp16) / 4 elements (fp32).
  *   - Notation: n1 = seq_len / segment_size, n2 = seq_len / block_size,
  *     r = segment_size / block_size (blocks that overlap a segment), k = budget_blocks,
  *     g = n_q_heads / n_kv_heads; query head h uses KV head h / g.
  *   - Requirements (else CP_ERR_SHAPE): seq_len % segment_size == 0,
  *     segment_size % block_size == 0, n_q_heads % n_kv_heads == 0, r <= k <= n2.
  *   - Supported (else CP_ERR_UNSUPPORTED): head_dim 64 or 128; n2 <= 8192 for estimate and select;
- *     the tensor-core attention path needs bf16, head_dim 128, segment_size % 256 == 0 and
+ *     the tensor-core attention path needs bf16 or fp16, head_dim 128, segment_size % 256 == 0 and
  *     block_size in {32, 64, 128}; everything else runs on a plain SIMT kernel.
  */
 #ifndef CRITIPREFILL_H_
@@ -51,7 +51,7 @@ typedef enum {
   CP_ERR_STATIC_LIMIT = 8 /* critiprefill_estimate_static: problem needs more scratch than the built-in array holds */
 } cp_status;
 
-typedef enum { CP_BF16 = 0, CP_F32 = 1 } cp_dtype;
+typedef enum { CP_BF16 = 0, CP_F32 = 1, CP_F16 = 2 } cp_dtype;   /* fp16 is the paper's own precision (Section 3.1.3) */
 
 enum {
   CP_FLAG_MASK_BEFORE_SOFTMAX = 1, /* estimate: normalise each score map over visible blocks only */
@@ -137,8 +137,8 @@ int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32
  *                  status block and its segment's rows of O are not written.
  *   O         out  device, same dtype and layout family as Q (o_stride)
  *   lse       out  device, nullable, [B,Hq,n] fp32: ln sum_{u in U_t} exp(sm_scale*q_t.k_u)
- * bf16: operands bf16, fp32 accumulation, probabilities rounded to bf16 before the PV
- * product, O rounded to bf16.  fp32: plain fp32 arithmetic. */
+ * bf16 / fp16: operands in that type, fp32 accumulation, probabilities rounded to that type
+ * before the PV product, O rounded to it.  fp32: plain fp32 arithmetic. */
 int critiprefill_attention(const cp_params* p, const void* Q, const void* K, const void* V,
                            const int32_t* idx, const int32_t* cnt, void* O, float* lse, void* ws,
                            size_t ws_bytes, void* cuda_stream);

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcritiprefill.so")
 
 CP_OK = 0
-CP_BF16, CP_F32 = 0, 1
+CP_BF16, CP_F32, CP_F16 = 0, 1, 2
 FLAG_MASK_BEFORE_SOFTMAX = 1
 FLAG_FORCE_SIMT = 2
 FLAG_TEST_WITHHOLD_V = 4
@@ -121,7 +121,8 @@ class Problem:
     @classmethod
     def from_config(cls, cfg, **kw) -> "Problem":
         return cls(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq_len, cfg.head_dim, cfg.segment_size,
-                   cfg.block_size, cfg.budget_blocks, torch.bfloat16 if cfg.dtype == "bf16" else torch.float32,
+                   cfg.block_size, cfg.budget_blocks,
+                   {"bf16": torch.bfloat16, "f32": torch.float32, "f16": torch.float16}[cfg.dtype],
                    est_scale=cfg.est_scale, alpha=cfg.alpha, **kw)
 
     @property
@@ -141,7 +142,7 @@ class Problem:
         p.batch, p.n_q_heads, p.n_kv_heads = self.batch, self.n_q_heads, self.n_kv_heads
         p.seq_len, p.head_dim = self.seq_len, self.head_dim
         p.segment_size, p.block_size, p.budget_blocks = self.segment_size, self.block_size, self.budget_blocks
-        p.dtype = CP_BF16 if self.dtype == torch.bfloat16 else CP_F32
+        p.dtype = {torch.bfloat16: CP_BF16, torch.float32: CP_F32, torch.float16: CP_F16}[self.dtype]
         p.flags = self.flags
         p.q_stride = _strides(Q) if Q is not None else self._contig(self.n_q_heads)
         p.k_stride = _strides(K) if K is not None else self._contig(self.n_kv_heads)

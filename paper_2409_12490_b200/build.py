@@ -28,7 +28,7 @@ def build(verbose: bool = False, force: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-           "--use_fast_math" if False else "-DCP_NO_FAST_MATH", "-Xcompiler", "-fPIC", "-shared",
+           "-Xcompiler", "-fPIC", "-shared",
            "-I", INCLUDE, "-I", CSRC, "-o", LIB] + sources()
     if verbose:
         cmd.insert(1, "-Xptxas")

@@ -19,7 +19,7 @@ class Config:
     n_kv_heads: int
     seq_len: int
     head_dim: int
-    dtype: str            # "bf16" | "f32"
+    dtype: str            # "bf16" | "f16" | "f32"
     segment_size: int
     block_size: int
     budget_tokens: int

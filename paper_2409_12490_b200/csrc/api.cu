@@ -10,7 +10,7 @@ int validate(const cp_params* p, Dims* out) {
   if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->seq_len <= 0 || p->head_dim <= 0 ||
       p->segment_size <= 0 || p->block_size <= 0 || p->budget_blocks <= 0)
     return CP_ERR_SHAPE;
-  if (p->dtype != CP_BF16 && p->dtype != CP_F32) return CP_ERR_UNSUPPORTED;
+  if (p->dtype != CP_BF16 && p->dtype != CP_F32 && p->dtype != CP_F16) return CP_ERR_UNSUPPORTED;
   if (p->n_q_heads % p->n_kv_heads) return CP_ERR_SHAPE;
   if (p->seq_len % p->segment_size || p->segment_size % p->block_size) return CP_ERR_SHAPE;
   Dims m = make_dims(*p);

@@ -13,7 +13,9 @@ constexpr int kWarps = 4;
 template <typename T> __device__ __forceinline__ float to_f32(T x);
 template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <> __device__ __forceinline__ float to_f32<__half>(__half x) { return __half2float(x); }
 template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ __half from_f32<__half>(float x) { return __float2half_rn(x); }
 template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
@@ -138,6 +140,9 @@ int launch_attention_simt(const cp_params& p, const Dims& m, const void* Q, cons
   if (p.dtype == CP_BF16) {
     if (m.d == 128) return launch_t<__nv_bfloat16, 128>(p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
     if (m.d == 64) return launch_t<__nv_bfloat16, 64>(p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
+  } else if (p.dtype == CP_F16) {
+    if (m.d == 128) return launch_t<__half, 128>(p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
+    if (m.d == 64) return launch_t<__half, 64>(p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
   } else {
     if (m.d == 128) return launch_t<float, 128>(p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);
     if (m.d == 64) return launch_t<float, 64>(p, m, Q, K, V, idx, cnt, O, lse, st, dense, s);

@@ -1,5 +1,5 @@
 // K4 / K5: block-sparse (Algorithm 2, lines 6-13) and dense causal (Eq. 2) attention on the
-// sm_100a tensor cores.  bf16 operands, fp32 accumulation in tensor memory, online softmax.
+// sm_100a tensor cores.  bf16 or fp16 operands, fp32 accumulation in tensor memory, online softmax.
 //
 // Persistent CTAs (one per SM) walk over work units; a unit is 256 consecutive query rows of one
 // (batch, query head): two 128-row tiles "A" and "B" that share every K/V tile the producer brings in.  Roles (384 threads):
@@ -56,7 +56,7 @@ struct Bars {
 struct Args {
   const int32_t* idx;
   const int32_t* cnt;
-  __nv_bfloat16* O;
+  uint16_t* O;                  // bf16 or fp16 elements
   float* lse;
   DeviceStatus* st;
   int B, Hq, Hkv, g, n, seg, blk, k, r, n1;
@@ -216,7 +216,12 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(r.y) << 23));
   return p;
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+template <bool kF16> __device__ __forceinline__ uint32_t pack2(float lo, float hi);   // two 16-bit values, `lo` in the low half
+template <> __device__ __forceinline__ uint32_t pack2<true>(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+template <> __device__ __forceinline__ uint32_t pack2<false>(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
@@ -232,8 +237,10 @@ __device__ __forceinline__ uint64_t desc_at(uint64_t base, uint32_t smem_addr) {
 
 // instruction descriptors: D fp32, A/B bf16, M = 128, N = 128; B is K-major for Q K^T and
 // MN-major (head_dim contiguous) for P V
-constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescPV = kIdescQK | (1u << 16);
+template <bool kF16> struct Idesc {   // operand format field: 0 = fp16, 1 = bf16
+  static constexpr uint32_t qk = (1u << 4) | ((kF16 ? 0u : 1u) << 7) | ((kF16 ? 0u : 1u) << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+  static constexpr uint32_t pv = qk | (1u << 16);
+};
 
 // ---------------------------------------------------------------- unit geometry
 struct Unit {
@@ -341,6 +348,7 @@ __device__ __forceinline__ int receive_unit(const Args& a, Bars* bars, uint32_t 
 // ---------------------------------------------------------------- softmax role
 constexpr int kMaskNone = 0, kMaskCausal = 1, kMaskCols = 2;
 
+template <bool kF16>
 __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int which, int warp_in_wg, int lane) {
   const uint32_t tm = bars->tmem_base;
   const uint32_t lane_off = uint32_t(warp_in_wg * 32) << 16;
@@ -361,7 +369,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     float m_run = -CUDART_INF, l_run = 0.f;
 
     for (int jt = 0; jt < my_tiles; ++jt, ++n_tiles) {
-      const bool tr = blockIdx.x == 0 && q == 0 && warp_in_wg == 0 && lane == 0 && jt < 64;
+      [[maybe_unused]] const bool tr = blockIdx.x == 0 && q == 0 && warp_in_wg == 0 && lane == 0 && jt < 64;
       CP_STAMP(tr, which * 1024 + jt * 8 + 0);
       if (!mbar_wait(&bars->s_full[which], n_tiles & 1, bars, a.st, 10 + which)) return;
       CP_STAMP(tr, which * 1024 + jt * 8 + 1);
@@ -425,7 +433,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
           if (kEmulEvery > 0 && (i >> 1) % kEmulEvery == kEmulEvery - 1) { p = exp2_poly2(xx); }
           else { p.x = ex2(xx.x); p.y = ex2(xx.y); }
           sum2 = __fadd2_rn(sum2, p);
-          pk[i >> 1] = pack_bf16(p.x, p.y);
+          pk[i >> 1] = pack2<kF16>(p.x, p.y);
         }
       } else {
 #pragma unroll
@@ -434,7 +442,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
           float2 p;
           p.x = ex2(xx.x); p.y = ex2(xx.y);
           sum2 = __fadd2_rn(sum2, p);
-          pk[i >> 1] = pack_bf16(p.x, p.y);
+          pk[i >> 1] = pack2<kF16>(p.x, p.y);
         }
       }
       l_run += sum2.x + sum2.y;
@@ -453,7 +461,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     ++n_units;
     tc_fence_after();
     const int t = u.q_tok + which * kTile + row;
-    __nv_bfloat16* orow = a.O + u.b * a.osb + u.h * a.osh + int64_t(t) * a.ost;
+    uint16_t* orow = a.O + u.b * a.osb + u.h * a.osh + int64_t(t) * a.ost;
     const float inv = 1.f / l_run;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -464,10 +472,10 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         uint4 w;
-        w.x = pack_bf16(__uint_as_float(ov[8 * i + 0]) * inv, __uint_as_float(ov[8 * i + 1]) * inv);
-        w.y = pack_bf16(__uint_as_float(ov[8 * i + 2]) * inv, __uint_as_float(ov[8 * i + 3]) * inv);
-        w.z = pack_bf16(__uint_as_float(ov[8 * i + 4]) * inv, __uint_as_float(ov[8 * i + 5]) * inv);
-        w.w = pack_bf16(__uint_as_float(ov[8 * i + 6]) * inv, __uint_as_float(ov[8 * i + 7]) * inv);
+        w.x = pack2<kF16>(__uint_as_float(ov[8 * i + 0]) * inv, __uint_as_float(ov[8 * i + 1]) * inv);
+        w.y = pack2<kF16>(__uint_as_float(ov[8 * i + 2]) * inv, __uint_as_float(ov[8 * i + 3]) * inv);
+        w.z = pack2<kF16>(__uint_as_float(ov[8 * i + 4]) * inv, __uint_as_float(ov[8 * i + 5]) * inv);
+        w.w = pack2<kF16>(__uint_as_float(ov[8 * i + 6]) * inv, __uint_as_float(ov[8 * i + 7]) * inv);
         dst[i] = w;
       }
     }
@@ -533,21 +541,24 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
 }
 
 // ---------------------------------------------------------------- MMA role
+template <bool kF16>
 __device__ __forceinline__ void issue_qk(uint32_t d_tmem, uint32_t q_smem, uint32_t k_smem) {
   const uint64_t base = desc_base(16);
 #pragma unroll
   for (int kk = 0; kk < kD / 16; ++kk) {
     const uint32_t off = (kk >> 2) * kHalfBytes + (kk & 3) * 32;
-    umma_ss(d_tmem, desc_at(base, q_smem + off), desc_at(base, k_smem + off), kIdescQK, kk > 0);
+    umma_ss(d_tmem, desc_at(base, q_smem + off), desc_at(base, k_smem + off), Idesc<kF16>::qk, kk > 0);
   }
 }
+template <bool kF16>
 __device__ __forceinline__ void issue_pv(uint32_t d_tmem, uint32_t p_tmem, uint32_t v_smem, bool acc) {
   const uint64_t base = desc_base(kHalfBytes);   // the two 64-column halves of head_dim are 16 KB apart
 #pragma unroll
   for (int kk = 0; kk < kTile / 16; ++kk)
-    umma_ts(d_tmem, p_tmem + kk * 8, desc_at(base, v_smem + kk * 16 * 128), kIdescPV, (acc || kk > 0) ? 1u : 0u);
+    umma_ts(d_tmem, p_tmem + kk * 8, desc_at(base, v_smem + kk * 16 * 128), Idesc<kF16>::pv, (acc || kk > 0) ? 1u : 0u);
 }
 
+template <bool kF16>
 __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t smem_base, int lane) {
   const uint32_t tm = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
   const uint32_t tS[2] = {tm, tm + 128}, tO[2] = {tm + 256, tm + 384};
@@ -569,8 +580,8 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
     if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;
     if (!full_wait(item0)) return;
     tc_fence_after();
-    issue_qk(tS[0], qA, slot_addr(item0)); umma_commit(&bars->s_full[0]);
-    issue_qk(tS[1], qB, slot_addr(item0)); umma_commit(&bars->s_full[1]);
+    issue_qk<kF16>(tS[0], qA, slot_addr(item0)); umma_commit(&bars->s_full[0]);
+    issue_qk<kF16>(tS[1], qB, slot_addr(item0)); umma_commit(&bars->s_full[1]);
     umma_commit(&bars->kv_empty[item0 % kSlots]);
     for (int jt = 0; jt < T; ++jt) {
       const bool has_next = jt + 1 < T;
@@ -578,15 +589,15 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
       if (has_next && !full_wait(ik)) return;
       if (!full_wait(iv)) return;
       const uint32_t v_smem = slot_addr(iv), kn_smem = slot_addr(ik);
-      const bool tr = blockIdx.x == 0 && q == 0 && lane == 0 && jt < 64;
+      [[maybe_unused]] const bool tr = blockIdx.x == 0 && q == 0 && lane == 0 && jt < 64;
       CP_STAMP(tr, 2048 + jt * 8 + 0);
       if (jt < TA) {
         if (!mbar_wait(&bars->p_full[0], nA & 1, bars, a.st, 42)) return;
         ++nA;
         CP_STAMP(tr, 2048 + jt * 8 + 1);
         tc_fence_after();
-        issue_pv(tO[0], tS[0], v_smem, jt > 0);
-        if (jt + 1 < TA) { issue_qk(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
+        issue_pv<kF16>(tO[0], tS[0], v_smem, jt > 0);
+        if (jt + 1 < TA) { issue_qk<kF16>(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
         else umma_commit(&bars->o_done[0]);
       }
       CP_STAMP(tr, 2048 + jt * 8 + 2);
@@ -594,10 +605,10 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
       ++nB;
       CP_STAMP(tr, 2048 + jt * 8 + 3);
       tc_fence_after();
-      issue_pv(tO[1], tS[1], v_smem, jt > 0);
+      issue_pv<kF16>(tO[1], tS[1], v_smem, jt > 0);
       umma_commit(&bars->kv_empty[iv % kSlots]);
       if (has_next) {
-        issue_qk(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
+        issue_qk<kF16>(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
         umma_commit(&bars->kv_empty[ik % kSlots]);
         if (jt + 1 == T - 1) umma_commit(&bars->q_empty);   // that was the unit's last QK^T: Q may be replaced
       } else {
@@ -611,6 +622,7 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
 }
 
 // ---------------------------------------------------------------- kernel
+template <bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKb,
                        const __grid_constant__ CUtensorMap tmVb, const __grid_constant__ CUtensorMap tmKt,
@@ -644,11 +656,11 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   static_assert(256 * 216 + 128 * 64 <= kThreads * 168, "setmaxnreg budget exceeds the launch allocation");
   if (warp < 8) {
     reg_inc<216>();
-    softmax_role(a, bars, warp >> 2, warp & 3, lane);
+    softmax_role<kF16>(a, bars, warp >> 2, warp & 3, lane);
   } else {
     reg_dec<64>();
     if (warp == 8) producer_role(a, bars, smem_base, &tmQ, &tmKb, &tmVb, &tmKt, &tmVt, lane);
-    else if (warp == 9) mma_role(a, bars, smem_base, lane);
+    else if (warp == 9) mma_role<kF16>(a, bars, smem_base, lane);
   }
   if (bars->abort_flag) {
     // give copies and MMAs still in flight time to land before the CTA's resources go away
@@ -678,14 +690,14 @@ EncodeTiledFn encode_fn() {
 }
 
 // [B, H, n, 128] bf16 with element strides (sb, sh, st); box = 64 columns x `rows` tokens
-bool make_map(CUtensorMap* map, const void* base, int B, int H, int n, const int64_t* s, int rows) {
+bool make_map(CUtensorMap* map, const void* base, int B, int H, int n, const int64_t* s, int rows, bool f16) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[4] = {cuuint64_t(kD), cuuint64_t(n), cuuint64_t(H), cuuint64_t(B)};
   cuuint64_t strides[3] = {cuuint64_t(s[2]) * 2, cuuint64_t(s[1]) * 2, cuuint64_t(s[0]) * 2};
   cuuint32_t box[4] = {64, cuuint32_t(rows), 1, 1};
   cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -693,7 +705,7 @@ bool make_map(CUtensorMap* map, const void* base, int B, int H, int n, const int
 }  // namespace
 
 bool sm100_path_applies(const cp_params& p, const Dims& m) {
-  return p.dtype == CP_BF16 && m.d == 128 && m.seg % 256 == 0 && (m.blk == 32 || m.blk == 64 || m.blk == 128) &&
+  return (p.dtype == CP_BF16 || p.dtype == CP_F16) && m.d == 128 && m.seg % 256 == 0 && (m.blk == 32 || m.blk == 64 || m.blk == 128) &&
          !(p.flags & CP_FLAG_FORCE_SIMT);
 }
 
@@ -701,19 +713,21 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
                            const int32_t* idx, const int32_t* cnt, void* O, float* lse, DeviceStatus* st,
                            bool dense, cudaStream_t s) {
   CUtensorMap tmQ, tmKb, tmVb, tmKt, tmVt;
-  if (!make_map(&tmQ, Q, m.B, m.Hq, m.n, p.q_stride, kTile) || !make_map(&tmKb, K, m.B, m.Hkv, m.n, p.k_stride, m.blk) ||
-      !make_map(&tmVb, V, m.B, m.Hkv, m.n, p.v_stride, m.blk) || !make_map(&tmKt, K, m.B, m.Hkv, m.n, p.k_stride, kTile) ||
-      !make_map(&tmVt, V, m.B, m.Hkv, m.n, p.v_stride, kTile))
+  const bool f16 = p.dtype == CP_F16;
+  if (!make_map(&tmQ, Q, m.B, m.Hq, m.n, p.q_stride, kTile, f16) || !make_map(&tmKb, K, m.B, m.Hkv, m.n, p.k_stride, m.blk, f16) ||
+      !make_map(&tmVb, V, m.B, m.Hkv, m.n, p.v_stride, m.blk, f16) || !make_map(&tmKt, K, m.B, m.Hkv, m.n, p.k_stride, kTile, f16) ||
+      !make_map(&tmVt, V, m.B, m.Hkv, m.n, p.v_stride, kTile, f16))
     return CP_ERR_CUDA;
   Args a;
-  a.idx = idx; a.cnt = cnt; a.O = static_cast<__nv_bfloat16*>(O); a.lse = lse; a.st = st;
+  a.idx = idx; a.cnt = cnt; a.O = static_cast<uint16_t*>(O); a.lse = lse; a.st = st;
   a.B = m.B; a.Hq = m.Hq; a.Hkv = m.Hkv; a.g = m.g; a.n = m.n; a.seg = m.seg; a.blk = m.blk; a.k = m.k;
   a.r = m.r; a.n1 = m.n1;
   a.osb = p.o_stride[0]; a.osh = p.o_stride[1]; a.ost = p.o_stride[2];
   a.sm_scale = p.sm_scale; a.dense = dense ? 1 : 0;
   const long long units = dense ? (long long)m.B * m.Hq * (m.n / 256) : (long long)m.B * m.Hq * m.n1 * (m.seg / 256);
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
-  if (cudaFuncSetAttribute(attention_sm100_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)
+  auto kern = f16 ? attention_sm100_kernel<true> : attention_sm100_kernel<false>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)
     return CP_ERR_CUDA;
   a.n_units = int(units);
   a.withhold_v = (p.flags & CP_FLAG_TEST_WITHHOLD_V) ? 1 : 0;
@@ -724,7 +738,7 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
     return CP_ERR_CUDA;
   // persistent CTAs, one per SM (the kernel takes all of an SM's tensor memory and shared memory)
   const unsigned grid = unsigned(units < sms ? units : sms);
-  attention_sm100_kernel<<<grid, kThreads, kSmemTotal, s>>>(tmQ, tmKb, tmVb, tmKt, tmVt, a);
+  kern<<<grid, kThreads, kSmemTotal, s>>>(tmQ, tmKb, tmVb, tmKt, tmVt, a);
   return check_launch();
 }
 

@@ -1,6 +1,7 @@
 // Shared host/device declarations of the CUDA path (not used by the CPU oracle).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -21,7 +22,7 @@ inline Dims make_dims(const cp_params& p) {
   m.B = p.batch; m.Hq = p.n_q_heads; m.Hkv = p.n_kv_heads; m.g = p.n_q_heads / p.n_kv_heads;
   m.n = p.seq_len; m.d = p.head_dim; m.seg = p.segment_size; m.blk = p.block_size;
   m.k = p.budget_blocks; m.n1 = p.seq_len / p.segment_size; m.n2 = p.seq_len / p.block_size;
-  m.r = p.segment_size / p.block_size; m.es = p.dtype == CP_BF16 ? 2 : 4;
+  m.r = p.segment_size / p.block_size; m.es = p.dtype == CP_F32 ? 4 : 2;
   return m;
 }
 

@@ -19,6 +19,7 @@ constexpr int kWarps = kThreads / 32;
 template <typename T> __device__ __forceinline__ double to_f64(T x);
 template <> __device__ __forceinline__ double to_f64<float>(float x) { return double(x); }
 template <> __device__ __forceinline__ double to_f64<__nv_bfloat16>(__nv_bfloat16 x) { return double(__bfloat162float(x)); }
+template <> __device__ __forceinline__ double to_f64<__half>(__half x) { return double(__half2float(x)); }
 
 // ln(e^a + e^b).  When the smaller term is more than e^-50 below the larger one it cannot change
 // the rounded result (|hi| is at most a few hundred here), so the transcendental pair is skipped.
@@ -235,6 +236,9 @@ int launch_score(const cp_params& p, const Dims& m, const char* ws, const double
   if (p.dtype == CP_BF16) {
     if (m.d == 128) return launch_t<__nv_bfloat16, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
     if (m.d == 64) return launch_t<__nv_bfloat16, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
+  } else if (p.dtype == CP_F16) {
+    if (m.d == 128) return launch_t<__half, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
+    if (m.d == 64) return launch_t<__half, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
   } else {
     if (m.d == 128) return launch_t<float, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
     if (m.d == 64) return launch_t<float, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);

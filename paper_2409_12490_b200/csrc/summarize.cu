@@ -17,7 +17,6 @@ constexpr int kThreads = kWarps * 32;
 template <typename T> struct Vec;
 template <> struct Vec<__nv_bfloat16> {
   uint4 v;
-  static constexpr int N = 4;  // packed words
   __device__ static Vec load(const void* p) { Vec r; r.v = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
   __device__ void store(void* p) const { *reinterpret_cast<uint4*>(p) = v; }
   __device__ static uint32_t mx(uint32_t a, uint32_t b) {
@@ -29,9 +28,21 @@ template <> struct Vec<__nv_bfloat16> {
     return *reinterpret_cast<uint32_t*>(&r);
   }
 };
+template <> struct Vec<__half> {
+  uint4 v;
+  __device__ static Vec load(const void* p) { Vec r; r.v = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
+  __device__ void store(void* p) const { *reinterpret_cast<uint4*>(p) = v; }
+  __device__ static uint32_t mx(uint32_t a, uint32_t b) {
+    __half2 r = __hmax2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+  }
+  __device__ static uint32_t mn(uint32_t a, uint32_t b) {
+    __half2 r = __hmin2(*reinterpret_cast<__half2*>(&a), *reinterpret_cast<__half2*>(&b));
+    return *reinterpret_cast<uint32_t*>(&r);
+  }
+};
 template <> struct Vec<float> {
   uint4 v;
-  static constexpr int N = 4;
   __device__ static Vec load(const void* p) { Vec r; r.v = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
   __device__ void store(void* p) const { *reinterpret_cast<uint4*>(p) = v; }
   __device__ static uint32_t mx(uint32_t a, uint32_t b) { return __float_as_uint(fmaxf(__uint_as_float(a), __uint_as_float(b))); }
@@ -68,7 +79,6 @@ struct Side {            // one tensor (Q or K) and where its summaries go
 template <typename T, int LPR>
 __device__ __forceinline__ void scan_rows(const char* gbase, int64_t st_bytes, int first, int nrows,
                                           int step, int lane, uint4& mx, uint4& mn) {
-  constexpr int RPW = 32 / LPR;               // rows per warp-wide load
   const int sub = lane / LPR, col = lane % LPR;
   const char* p0 = gbase + int64_t(first + sub) * st_bytes + col * 16;
   bool init = false;
@@ -88,7 +98,6 @@ __device__ __forceinline__ void scan_rows(const char* gbase, int64_t st_bytes, i
     if (!init) { mx = v; mn = v; init = true; }
     vmax<T>(mx, v); vmin<T>(mn, v);
   }
-  (void)RPW;
 }
 
 template <typename T, int LPR>
@@ -182,6 +191,9 @@ int launch_summarize(const cp_params& p, const Dims& m, const void* Q, const voi
   if (p.dtype == CP_BF16) {
     if (lpr == 16) return launch_t<__nv_bfloat16, 16>(q, k, ctas, m.d, st);
     if (lpr == 8) return launch_t<__nv_bfloat16, 8>(q, k, ctas, m.d, st);
+  } else if (p.dtype == CP_F16) {
+    if (lpr == 16) return launch_t<__half, 16>(q, k, ctas, m.d, st);
+    if (lpr == 8) return launch_t<__half, 8>(q, k, ctas, m.d, st);
   } else {
     if (lpr == 32) return launch_t<float, 32>(q, k, ctas, m.d, st);
     if (lpr == 16) return launch_t<float, 16>(q, k, ctas, m.d, st);

@@ -45,7 +45,7 @@ def _ar1(x: np.ndarray, rho: float) -> np.ndarray:
 
 def _to_storage(x: np.ndarray, dtype: str) -> torch.Tensor:
     t = torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32))
-    return t.to(torch.bfloat16) if dtype == "bf16" else t
+    return t.to({"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype])
 
 
 def make_qkv(cfg: Config, layer: int = 0, threads: int = 8):
@@ -53,7 +53,7 @@ def make_qkv(cfg: Config, layer: int = 0, threads: int = 8):
     B, Hq, Hkv, n, d = cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.seq_len, cfg.head_dim
     g = Hq // Hkv
     seed = BASE_SEED + 1000 * cfg.index + layer
-    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[cfg.dtype]
     Q = torch.empty((B, Hq, n, d), dtype=tdt)
     K = torch.empty((B, Hkv, n, d), dtype=tdt)
     V = torch.empty((B, Hkv, n, d), dtype=tdt)

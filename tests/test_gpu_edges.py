@@ -139,3 +139,20 @@ def test_host_pipelined_layer_equals_resident_path():
     torch.cuda.synchronize()
     assert layer.status() == 0 and cp.device_status(ws) == 0
     assert torch.equal(hO, O_res.cpu())
+
+
+@pytest.mark.parametrize("flags", [0, cp.FLAG_FORCE_SIMT])
+def test_fp16_inputs_whole_path(flags):
+    """fp16 is the precision the paper ran in (Section 3.1.3): same path, same oracle, same bounds."""
+    cfg = CONFIGS["C2"].with_(name="half", dtype="f16", seq_len=2048, n_q_heads=4, n_kv_heads=2, segment_size=256,
+                              block_size=64, budget_tokens=512, n_clusters=16)
+    Q, K, V = make_qkv(cfg)
+    assert Q.dtype == torch.float16
+    O = full_path_vs_oracle(cfg, Q, K, V, flags=flags)
+    assert O.dtype == torch.float16
+    prob = problem(cfg, flags=flags)
+    ws = cp.alloc_workspace(prob)
+    Od = cp.dense_attention(prob, *to_dev(Q, K, V), ws)
+    assert cp.device_status(ws) == 0
+    O_ref, _ = oracle.dense_attention(Q, K, V, f32(1.0 / np.sqrt(cfg.head_dim)))
+    assert_attention_close(Od, O_ref)
