@@ -26,7 +26,7 @@
  *   - Requirements (else CP_ERR_SHAPE): seq_len % segment_size == 0,
  *     segment_size % block_size == 0, n_q_heads % n_kv_heads == 0, r <= k <= n2.
  *   - Supported (else CP_ERR_UNSUPPORTED): head_dim 64 or 128; n2 <= 8192 for estimate and select;
- *     the tensor-core attention path needs bf16 or fp16, head_dim 128, segment_size % 256 == 0 and
+ *     the tensor-core attention path needs bf16 or fp16, head_dim 128, segment_size % 128 == 0 and
  *     block_size in {32, 64, 128}; everything else runs on a plain SIMT kernel.
  */
 #ifndef CRITIPREFILL_H_

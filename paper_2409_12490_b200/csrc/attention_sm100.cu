@@ -2,7 +2,8 @@
 // sm_100a tensor cores.  bf16 or fp16 operands, fp32 accumulation in tensor memory, online softmax.
 //
 // Persistent CTAs (one per SM) walk over work units; a unit is 256 consecutive query rows of one
-// (batch, query head): two 128-row tiles "A" and "B" that share every K/V tile the producer brings in.  Roles (384 threads):
+// (batch, query head): two 128-row tiles "A" and "B" that share every K/V tile the producer brings in
+// (tile B is absent in the last unit of a segment with an odd number of 128-row tiles).  Roles (384 threads):
 //   warps 0-3  softmax for tile A (one thread per query row)
 //   warps 4-7  softmax for tile B
 //   warp  8    TMA producer: K/V tiles through a 5-slot ring of 32 KB buffers; a gathered
@@ -251,7 +252,8 @@ struct Unit {
   int last_cols;    // valid key columns of the last gathered tile
   int c_tok, n_cont;// contiguous unmasked tiles: first token, count
   int d_tok;        // first token of diagonal tile d0 (d1 follows)
-  int T;            // tiles for B; A takes T-1
+  int T;            // K/V tiles the unit streams
+  int nA, nB;       // tiles query tile A / B consumes (nB = 0: the unit has no tile B)
   const int32_t* list;
   int seg_j;
   int cnt;
@@ -264,7 +266,8 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
   u.list = nullptr;
   u.cnt = 0;
   if (a.dense) {
-    const int np = a.n / 256;
+    const int ntiles = a.n / kTile;
+    const int np = (ntiles + 1) / 2;
     const int per_kvh = a.g * np;
     const int bkv = x / per_kvh;
     const int rest = x - bkv * per_kvh;
@@ -275,8 +278,10 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
     u.n_past = 0; u.n_past_tiles = 0; u.last_cols = kTile;
     u.c_tok = 0; u.n_cont = 2 * pair; u.d_tok = pair * 256;
     u.seg_j = 0;
+    u.nB = (2 * pair + 1 < ntiles) ? 1 : 0;
   } else {
-    const int pp = a.seg / 256;
+    const int q_tiles = a.seg / kTile;
+    const int pp = (q_tiles + 1) / 2;
     const int gi_p = a.g * pp;
     const int per_kvh = a.n1 * gi_p;
     const int bkv = x / per_kvh;
@@ -294,8 +299,11 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
     u.n_past_tiles = (u.n_past * a.blk + kTile - 1) / kTile;
     u.last_cols = u.n_past * a.blk - (u.n_past_tiles - 1) * kTile;
     u.c_tok = j * a.seg; u.n_cont = 2 * p; u.d_tok = u.q_tok;
+    u.nB = (2 * p + 1 < q_tiles) ? 1 : 0;
   }
-  u.T = u.n_past_tiles + u.n_cont + 2;
+  u.nA = u.n_past_tiles + u.n_cont + 1;       // up to and including its own diagonal tile
+  u.nB = u.nB ? u.nA + 1 : 0;                 // one more diagonal tile; 0 when the segment has an odd tile count
+  u.T = u.nB ? u.nB : u.nA;
   return u;
 }
 
@@ -365,7 +373,8 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     if (!got || x >= a.n_units || stop_requested(a, bars)) return;
     const Unit u = decode_unit(a, x);
     if (!unit_ok(a, u, lane)) continue;
-    const int my_tiles = which == 0 ? u.T - 1 : u.T;
+    const int my_tiles = which == 0 ? u.nA : u.nB;
+    if (my_tiles == 0) continue;                        // this unit has no tile B
     float m_run = -CUDART_INF, l_run = 0.f;
 
     for (int jt = 0; jt < my_tiles; ++jt, ++n_tiles) {
@@ -503,8 +512,9 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
     // Q tiles: the buffer is free once every QK^T of the previous unit has completed
     if (n_units > 0 && !mbar_wait(&bars->q_empty, (n_units - 1) & 1, bars, a.st, 31)) return;
     if (lane == 0) {
-      mbar_expect_tx(&bars->q_full, 2 * kTileBytes);
-      for (int w = 0; w < 2; ++w)
+      const int nq = u.nB ? 2 : 1;
+      mbar_expect_tx(&bars->q_full, nq * kTileBytes);
+      for (int w = 0; w < nq; ++w)
         for (int hf = 0; hf < 2; ++hf)
           tma_load_4d(smem_base + kSmemQ + w * kTileBytes + hf * kHalfBytes, tmQ, &bars->q_full, hf * 64,
                       u.q_tok + w * kTile, u.h, u.b);
@@ -576,13 +586,15 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
     if (!got || x >= a.n_units || stop_requested(a, bars)) return;
     const Unit u = decode_unit(a, x);
     if (!unit_ok(a, u, lane)) continue;
-    const int T = u.T, TA = u.T - 1;
+    const int T = u.T, TA = u.nA;
+    const bool hasB = u.nB > 0;
     if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;
     if (!full_wait(item0)) return;
     tc_fence_after();
     issue_qk<kF16>(tS[0], qA, slot_addr(item0)); umma_commit(&bars->s_full[0]);
-    issue_qk<kF16>(tS[1], qB, slot_addr(item0)); umma_commit(&bars->s_full[1]);
+    if (hasB) { issue_qk<kF16>(tS[1], qB, slot_addr(item0)); umma_commit(&bars->s_full[1]); }
     umma_commit(&bars->kv_empty[item0 % kSlots]);
+    if (T == 1) umma_commit(&bars->q_empty);               // a one-tile unit has no further QK^T
     for (int jt = 0; jt < T; ++jt) {
       const bool has_next = jt + 1 < T;
       const uint32_t iv = item0 + 2 * jt + 1, ik = item0 + 2 * (jt + 1);
@@ -601,17 +613,19 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
         else umma_commit(&bars->o_done[0]);
       }
       CP_STAMP(tr, 2048 + jt * 8 + 2);
-      if (!mbar_wait(&bars->p_full[1], nB & 1, bars, a.st, 43)) return;
-      ++nB;
-      CP_STAMP(tr, 2048 + jt * 8 + 3);
-      tc_fence_after();
-      issue_pv<kF16>(tO[1], tS[1], v_smem, jt > 0);
-      umma_commit(&bars->kv_empty[iv % kSlots]);
+      if (hasB) {
+        if (!mbar_wait(&bars->p_full[1], nB & 1, bars, a.st, 43)) return;
+        ++nB;
+        CP_STAMP(tr, 2048 + jt * 8 + 3);
+        tc_fence_after();
+        issue_pv<kF16>(tO[1], tS[1], v_smem, jt > 0);
+      }
+      umma_commit(&bars->kv_empty[iv % kSlots]);             // every PV that reads this V tile has been issued
       if (has_next) {
-        issue_qk<kF16>(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]);
+        if (hasB) { issue_qk<kF16>(tS[1], qB, kn_smem); umma_commit(&bars->s_full[1]); }
         umma_commit(&bars->kv_empty[ik % kSlots]);
         if (jt + 1 == T - 1) umma_commit(&bars->q_empty);   // that was the unit's last QK^T: Q may be replaced
-      } else {
+      } else if (hasB) {
         umma_commit(&bars->o_done[1]);
       }
       CP_STAMP(tr, 2048 + jt * 8 + 4);
@@ -705,7 +719,7 @@ bool make_map(CUtensorMap* map, const void* base, int B, int H, int n, const int
 }  // namespace
 
 bool sm100_path_applies(const cp_params& p, const Dims& m) {
-  return (p.dtype == CP_BF16 || p.dtype == CP_F16) && m.d == 128 && m.seg % 256 == 0 && (m.blk == 32 || m.blk == 64 || m.blk == 128) &&
+  return (p.dtype == CP_BF16 || p.dtype == CP_F16) && m.d == 128 && m.seg % kTile == 0 && (m.blk == 32 || m.blk == 64 || m.blk == 128) &&
          !(p.flags & CP_FLAG_FORCE_SIMT);
 }
 
@@ -724,7 +738,9 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
   a.r = m.r; a.n1 = m.n1;
   a.osb = p.o_stride[0]; a.osh = p.o_stride[1]; a.ost = p.o_stride[2];
   a.sm_scale = p.sm_scale; a.dense = dense ? 1 : 0;
-  const long long units = dense ? (long long)m.B * m.Hq * (m.n / 256) : (long long)m.B * m.Hq * m.n1 * (m.seg / 256);
+  // a unit is two 128-row query tiles (one when a segment, or the sequence, has an odd tile count)
+  const long long units = dense ? (long long)m.B * m.Hq * ((m.n / kTile + 1) / 2)
+                                : (long long)m.B * m.Hq * m.n1 * ((m.seg / kTile + 1) / 2);
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
   auto kern = f16 ? attention_sm100_kernel<true> : attention_sm100_kernel<false>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)

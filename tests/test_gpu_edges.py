@@ -67,10 +67,20 @@ def test_large_logits_exercise_the_rescale_path():
     assert mx <= bound and mean <= TOL_BF16_MEAN, (mx, mean, bound)
 
 
-@pytest.mark.parametrize("seg,blk,d", [(128, 32, 128), (384, 64, 128), (256, 64, 64)])
-def test_shapes_served_by_the_simt_kernel(seg, blk, d):
-    cfg = BASE.with_(seq_len=768, segment_size=seg, block_size=blk, budget_tokens=max(seg, 256), head_dim=d)
-    full_path_vs_oracle(cfg, *make_qkv(cfg))
+@pytest.mark.parametrize("n,seg,blk,d", [(768, 128, 32, 128), (768, 384, 64, 128), (1280, 640, 128, 128),
+                                         (640, 128, 128, 128), (768, 256, 64, 64)])
+def test_odd_tile_counts_and_simt_shapes(n, seg, blk, d):
+    """Segments of 1, 3 or 5 query tiles (the last work unit of a segment then has a single tile), a
+    sequence of 5 tiles for the dense kernel, and head_dim 64, which the SIMT kernel serves."""
+    cfg = BASE.with_(seq_len=n, segment_size=seg, block_size=blk, budget_tokens=max(seg, 256), head_dim=d)
+    Q, K, V = make_qkv(cfg)
+    full_path_vs_oracle(cfg, Q, K, V)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Od = cp.dense_attention(prob, *to_dev(Q, K, V), ws)
+    assert cp.device_status(ws) == 0
+    O_ref, _ = oracle.dense_attention(Q, K, V, f32(1.0 / np.sqrt(cfg.head_dim)))
+    assert_attention_close(Od, O_ref)
 
 
 def test_fp32_path_with_strided_output():
