@@ -76,7 +76,10 @@ typedef struct {
 
 /* Bytes of scratch (`ws`) the calls below need for these parameters; the same buffer serves
  * all of them.  `ws` must be 256-byte aligned.  Its first 256 bytes are the device status
- * block, which the caller zeroes once (cudaMemset) before the first call.  Host pointers. */
+ * block, which the caller zeroes once (cudaMemset) before the first call; the attention calls
+ * also keep their work-unit counter there and reset it themselves at every launch.  Calls that
+ * may execute concurrently (different streams without ordering) need separate workspaces;
+ * calls ordered on one stream can share one.  Host pointers. */
 int critiprefill_workspace_bytes(const cp_params* p, size_t* bytes_out);
 
 /* Algorithm 1 (estimation of query criticality in one layer).
