@@ -8,11 +8,13 @@
 //   warps 4-7  softmax for tile B
 //   warp  8    TMA producer: K/V tiles through a 5-slot ring of 32 KB buffers; a gathered
 //              tile is assembled from 128/blk boxes addressed by the block list
-//   warp  9    MMA issuer (warps 10-11 idle; they complete the third warpgroup): S = Q K^T (operands in shared memory), O += P V (P read from
-//              tensor memory, where the softmax warps overwrite S with bf16 probabilities)
+//   warp  9    MMA issuer (warps 10-11 idle; they complete the third warpgroup): S = Q K^T
+//              (operands in shared memory), O += P V (P read from tensor memory, where the
+//              softmax warps overwrite S with 16-bit probabilities)
 // Tensor memory (512 columns): S_A | S_B | O_A | O_B, 128 fp32 columns each.
 // The tile sequence of a unit is: gathered past tiles, contiguous unmasked tiles, then the
-// two diagonal tiles; tile A stops one tile earlier than B.  Every wait is bounded: on
+// diagonal tiles; tile A stops one tile earlier than B.  Units are handed out by an atomic
+// counter (producer warp) and published to the other warps.  Every wait is bounded: on
 // expiry the waiter raises a CTA-wide abort flag and CP_ERR_TIMEOUT, and all roles drain.
 #include <cuda.h>
 #include <math_constants.h>
@@ -24,14 +26,14 @@ namespace {
 
 constexpr int kD = 128;
 constexpr int kTile = 128;
-constexpr int kHalfBytes = kTile * 64 * 2;   // [128 rows x 64 cols] bf16, 128-byte swizzled
+constexpr int kHalfBytes = kTile * 64 * 2;   // [128 rows x 64 cols] of 16-bit elements, 128-byte swizzled
 constexpr int kTileBytes = 2 * kHalfBytes;   // both halves of head_dim
 constexpr int kSlots = 5;
 constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer, MMA, 2 idle}
 constexpr int kSmemQ = 0;
 constexpr int kSmemKV = 2 * kTileBytes;
 constexpr int kSmemBar = kSmemKV + kSlots * kTileBytes;
-constexpr int kSmemTotal = kSmemBar + 256 + 1024;   // + alignment slack
+constexpr int kSmemTotal = kSmemBar + 256 + 1024;   // + barrier block + slack to align the tiles to 1024 bytes
 constexpr float kRescaleThreshold = 8.0f;           // in log2 units
 #ifndef CP_EMUL_EVERY
 #define CP_EMUL_EVERY 4
