@@ -52,6 +52,7 @@ struct Bars {
   unsigned long long sched_full[2];
   unsigned long long sched_empty[2];
   int sched_unit[2];
+  int sched_cnt[2];
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -263,7 +264,9 @@ struct Unit {
 
 // Units are ordered KV-head-major so that CTAs resident at the same time share K/V tiles in
 // L2; within a KV head the dense kernel takes the longest rows first.
-__device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
+// `cnt` is the unit's list length when the caller already has it, kLoadCnt to read it from global memory.
+constexpr int kLoadCnt = -2, kBadList = -1;
+__device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
   Unit u;
   u.list = nullptr;
   u.cnt = 0;
@@ -296,7 +299,7 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
     u.q_tok = j * a.seg + p * 256;
     const long long unit = ((long long)u.b * a.Hq + u.h) * a.n1 + j;
     u.list = a.idx + unit * a.k;
-    u.cnt = a.cnt[unit];
+    u.cnt = cnt == kLoadCnt ? a.cnt[unit] : cnt;
     u.n_past = min(max(u.cnt - a.r, 0), a.k);
     u.n_past_tiles = (u.n_past * a.blk + kTile - 1) / kTile;
     u.last_cols = u.n_past * a.blk - (u.n_past_tiles - 1) * kTile;
@@ -309,9 +312,8 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x) {
   return u;
 }
 
-// The list contract, checked by every warp for itself (all warps reach the same verdict, so
-// no CTA-wide synchronisation is needed): r <= cnt <= k, ascending past blocks, then exactly
-// the r diagonal blocks of the segment.
+// The list contract, checked by the producer warp before it publishes a unit: r <= cnt <= k,
+// ascending past blocks, then exactly the r diagonal blocks of the segment.
 __device__ __forceinline__ bool unit_ok(const Args& a, const Unit& u, int lane) {
   if (a.dense) return true;
   bool ok = (u.cnt >= a.r) && (u.cnt <= a.k);
@@ -331,28 +333,42 @@ __device__ __forceinline__ bool stop_requested(const Args& a, Bars* bars) {
 
 // ---------------------------------------------------------------- unit scheduler
 // Units are handed out dynamically (an atomic counter in global memory) so that SMs that run
-// faster take more of them.  The producer warp draws the q-th unit of this CTA and publishes
-// it through a two-entry ring; the MMA warp and the eight softmax warps read it from there.
-__device__ __forceinline__ int publish_unit(const Args& a, Bars* bars, uint32_t q, int lane, bool* ok) {
+// faster take more of them.  The producer warp draws the q-th unit of this CTA, reads and checks
+// its block list, and publishes (unit, list length) through a two-entry ring; the MMA warp and
+// the eight softmax warps take it from there and touch no global memory at a unit's start.
+// A list that breaks its contract is published with length kBadList and skipped by everyone.
+__device__ __forceinline__ bool publish_unit(const Args& a, Bars* bars, uint32_t q, int lane, int* x_out, Unit* u_out) {
   const uint32_t slot = q & 1;
-  *ok = true;
-  if (q >= 2 && !mbar_wait(&bars->sched_empty[slot], ((q >> 1) - 1) & 1, bars, a.st, 50)) { *ok = false; return 0; }
+  if (q >= 2 && !mbar_wait(&bars->sched_empty[slot], ((q >> 1) - 1) & 1, bars, a.st, 50)) return false;
   int x = 0;
+  if (lane == 0) x = int(min(atomicAdd(a.work_counter, 1u), 0x7fffffffu));
+  x = __shfl_sync(0xffffffffu, x, 0);
+  int cnt = 0;
+  if (x < a.n_units) {
+    *u_out = decode_unit(a, x, kLoadCnt);
+    cnt = u_out->cnt;
+    if (!unit_ok(a, *u_out, lane)) {
+      if (lane == 0) report(a.st, CP_ERR_BOUNDS, 1, u_out->b, u_out->h, u_out->seg_j, u_out->cnt);
+      cnt = kBadList;
+    }
+  }
   if (lane == 0) {
-    x = int(min(atomicAdd(a.work_counter, 1u), 0x7fffffffu));
     bars->sched_unit[slot] = x;
+    bars->sched_cnt[slot] = cnt;
     mbar_arrive(&bars->sched_full[slot]);
   }
-  return __shfl_sync(0xffffffffu, x, 0);
+  *x_out = x;
+  u_out->cnt = cnt;
+  return true;
 }
-__device__ __forceinline__ int receive_unit(const Args& a, Bars* bars, uint32_t q, int lane, bool* ok) {
+__device__ __forceinline__ bool receive_unit(const Args& a, Bars* bars, uint32_t q, int lane, int* x_out, int* cnt_out) {
   const uint32_t slot = q & 1;
-  *ok = mbar_wait(&bars->sched_full[slot], (q >> 1) & 1, bars, a.st, 51);
-  if (!*ok) return 0;
-  const int x = *reinterpret_cast<volatile int*>(&bars->sched_unit[slot]);
+  if (!mbar_wait(&bars->sched_full[slot], (q >> 1) & 1, bars, a.st, 51)) return false;
+  *x_out = *reinterpret_cast<volatile int*>(&bars->sched_unit[slot]);
+  *cnt_out = *reinterpret_cast<volatile int*>(&bars->sched_cnt[slot]);
   __syncwarp();
   if (lane == 0) mbar_arrive(&bars->sched_empty[slot]);
-  return x;
+  return true;
 }
 
 // ---------------------------------------------------------------- softmax role
@@ -370,11 +386,10 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
   uint32_t n_units = 0;                               // units finished so far
 
   for (uint32_t q = 0;; ++q) {
-    bool got;
-    const int x = receive_unit(a, bars, q, lane, &got);
-    if (!got || x >= a.n_units || stop_requested(a, bars)) return;
-    const Unit u = decode_unit(a, x);
-    if (!unit_ok(a, u, lane)) continue;
+    int x, cnt;
+    if (!receive_unit(a, bars, q, lane, &x, &cnt) || x >= a.n_units || stop_requested(a, bars)) return;
+    if (cnt == kBadList) continue;
+    const Unit u = decode_unit(a, x, cnt);
     const int my_tiles = which == 0 ? u.nA : u.nB;
     if (my_tiles == 0) continue;                        // this unit has no tile B
     float m_run = -CUDART_INF, l_run = 0.f;
@@ -502,27 +517,28 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
   const int bpt = kTile / a.blk;
   uint32_t item = 0;      // K/V tiles issued so far (all units): item i lives in slot i % kSlots
   uint32_t n_units = 0;
+  // One unit of look-ahead: unit q+1 is drawn, checked and published before the loads of unit q
+  // are issued, so the other warps never wait for the counter or for the list to be read.
+  int x;
+  Unit u;
+  if (!publish_unit(a, bars, 0, lane, &x, &u)) return;
   for (uint32_t q = 0;; ++q) {
-    bool got;
-    const int x = publish_unit(a, bars, q, lane, &got);
-    if (!got || x >= a.n_units || stop_requested(a, bars)) return;
-    const Unit u = decode_unit(a, x);
-    if (!unit_ok(a, u, lane)) {
-      if (lane == 0) report(a.st, CP_ERR_BOUNDS, 1, u.b, u.h, u.seg_j, u.cnt);
-      continue;
-    }
+    if (x >= a.n_units || stop_requested(a, bars)) return;
+    const Unit u_cur = u;
+    if (!publish_unit(a, bars, q + 1, lane, &x, &u)) return;
+    if (u_cur.cnt == kBadList) continue;
     // Q tiles: the buffer is free once every QK^T of the previous unit has completed
     if (n_units > 0 && !mbar_wait(&bars->q_empty, (n_units - 1) & 1, bars, a.st, 31)) return;
     if (lane == 0) {
-      const int nq = u.nB ? 2 : 1;
+      const int nq = u_cur.nB ? 2 : 1;
       mbar_expect_tx(&bars->q_full, nq * kTileBytes);
       for (int w = 0; w < nq; ++w)
         for (int hf = 0; hf < 2; ++hf)
           tma_load_4d(smem_base + kSmemQ + w * kTileBytes + hf * kHalfBytes, tmQ, &bars->q_full, hf * 64,
-                      u.q_tok + w * kTile, u.h, u.b);
+                      u_cur.q_tok + w * kTile, u_cur.h, u_cur.b);
     }
     ++n_units;
-    for (int it = 0; it < 2 * u.T; ++it, ++item) {   // 2*jt = K tile jt, 2*jt+1 = V tile jt
+    for (int it = 0; it < 2 * u_cur.T; ++it, ++item) {   // 2*jt = K tile jt, 2*jt+1 = V tile jt
       const uint32_t slot = item % kSlots, use = item / kSlots;
       if (use > 0 && !mbar_wait(&bars->kv_empty[slot], (use - 1) & 1, bars, a.st, 30)) return;
       if (lane == 0 && !(a.withhold_v && (it & 1))) {
@@ -531,20 +547,20 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
         const uint32_t dst = smem_base + kSmemKV + slot * kTileBytes;
         unsigned long long* bar = &bars->kv_full[slot];
         mbar_expect_tx(bar, kTileBytes);
-        if (jt < u.n_past_tiles) {
+        if (jt < u_cur.n_past_tiles) {
           const CUtensorMap* tm = is_v ? tmVb : tmKb;
           for (int q = 0; q < bpt; ++q) {
             const int li = jt * bpt + q;
             // boxes beyond the list read past the end of the tensor and arrive as zeros
-            const int tok = li < u.n_past ? u.list[li] * a.blk : a.n;
+            const int tok = li < u_cur.n_past ? u_cur.list[li] * a.blk : a.n;
             for (int hf = 0; hf < 2; ++hf)
-              tma_load_4d(dst + hf * kHalfBytes + q * a.blk * 128, tm, bar, hf * 64, tok, u.kvh, u.b);
+              tma_load_4d(dst + hf * kHalfBytes + q * a.blk * 128, tm, bar, hf * 64, tok, u_cur.kvh, u_cur.b);
           }
         } else {
           const CUtensorMap* tm = is_v ? tmVt : tmKt;
-          const int ci = jt - u.n_past_tiles;
-          const int tok = ci < u.n_cont ? u.c_tok + ci * kTile : u.d_tok + (ci - u.n_cont) * kTile;
-          for (int hf = 0; hf < 2; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, bar, hf * 64, tok, u.kvh, u.b);
+          const int ci = jt - u_cur.n_past_tiles;
+          const int tok = ci < u_cur.n_cont ? u_cur.c_tok + ci * kTile : u_cur.d_tok + (ci - u_cur.n_cont) * kTile;
+          for (int hf = 0; hf < 2; ++hf) tma_load_4d(dst + hf * kHalfBytes, tm, bar, hf * 64, tok, u_cur.kvh, u_cur.b);
         }
       }
       __syncwarp();
@@ -583,11 +599,10 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
     return mbar_wait(&bars->kv_full[item % kSlots], (item / kSlots) & 1, bars, a.st, 40);
   };
   for (uint32_t q = 0;; ++q) {
-    bool got;
-    const int x = receive_unit(a, bars, q, lane, &got);
-    if (!got || x >= a.n_units || stop_requested(a, bars)) return;
-    const Unit u = decode_unit(a, x);
-    if (!unit_ok(a, u, lane)) continue;
+    int x, cnt;
+    if (!receive_unit(a, bars, q, lane, &x, &cnt) || x >= a.n_units || stop_requested(a, bars)) return;
+    if (cnt == kBadList) continue;
+    const Unit u = decode_unit(a, x, cnt);
     const int T = u.T, TA = u.nA;
     const bool hasB = u.nB > 0;
     if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;
