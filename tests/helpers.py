@@ -78,7 +78,7 @@ def assert_attention_close(O_gpu, O_ref, tol_max=TOL_BF16_MAX, tol_mean=TOL_BF16
     values.  Outputs are stored in bf16, whose spacing is 2^-6 for 2 <= |O| < 4 and 2^-5 beyond, so an
     absolute 1e-2 is not attainable there even with exact arithmetic; for |O_ref| >= 2 the bound is
     therefore relative, 1e-2 * |O_ref|.  Returns (max abs err where |O_ref| < 2, mean abs err,
-    number of elements judged by the relative bound)."""
+    number of elements checked against the relative bound)."""
     O = O_gpu.float().cpu().numpy().astype(np.float64) if hasattr(O_gpu, "cpu") else np.asarray(O_gpu, dtype=np.float64)
     err = np.abs(O - O_ref)
     big = np.abs(O_ref) >= 2.0

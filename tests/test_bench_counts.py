@@ -1,5 +1,5 @@
 """The roofline numerator: bench.flop_counts must equal an explicit enumeration of the (query tile,
-KV tile) pairs the sparse kernel issues, and the analytic totals of the survey table."""
+KV tile) pairs the sparse kernel issues, and the analytic totals (full listed tiles, causal-useful, dense)."""
 import importlib.util
 import os
 
@@ -36,7 +36,7 @@ def test_executed_flops_match_tile_enumeration():
         assert fl["useful"] <= fl["executed"] <= fl["listed_full_tiles"]
 
 
-def test_survey_totals_at_c4():
+def test_analytic_totals_at_c4():
     fl = bench.flop_counts(CONFIGS["C4"])
     assert abs(fl["listed_full_tiles"] / 1e12 - 8.693) < 1e-3      # every listed block against its whole segment
     assert abs(fl["useful"] / 1e12 - 7.595) < 1e-3
