@@ -58,7 +58,7 @@ def _rows(Q, K, V, idx, cnt, seg, blk, k, sm_scale, rows):
     if idx is not None:
         idx = np.ascontiguousarray(idx, dtype=np.int32)
         cnt = np.ascontiguousarray(cnt, dtype=np.int32)
-        assert idx.shape == (B, Hq, n // seg, k) and cnt.shape == (B, Hq, n // seg)
+        assert idx.shape == (B, Hq, -(-n // seg), k) and cnt.shape == (B, Hq, -(-n // seg))
     err = _lib().oracle_attention_rows(
         P(Q.ctypes.data), P(K.ctypes.data), P(V.ctypes.data),
         P(idx.ctypes.data) if idx is not None else P(0), P(cnt.ctypes.data) if idx is not None else P(0),

@@ -49,7 +49,7 @@ int oracle_attention_rows(const float *Q, const float *K, const float *V,
 {
     (void)B;
     int g = Hq / Hkv;
-    int64_t n1 = n / seg;
+    int64_t n1 = (n + seg - 1) / seg;   /* the last segment may be shorter */
     int err = 0;
 #pragma omp parallel
     {

@@ -20,7 +20,9 @@ among them is "parity unpinned" with respect to the authors' implementation):
     ``mask_before_softmax`` gives the other order;
   * a block is masked iff it starts at or after the end of the segment;
   * every query head has its own score map, using the key summaries of its KV group;
-  * S' = None means no fusion; the fused S is what the next layer receives.
+  * S' = None means no fusion; the fused S is what the next layer receives;
+  * a sequence length that is not a multiple of the segment / block size leaves a shorter last
+    segment / block (n1 = ceil(n/seg), n2 = ceil(n/blk)); the paper writes the divisions as exact.
 """
 from __future__ import annotations
 
@@ -44,11 +46,16 @@ def summaries(Q, K, segment_size: int, block_size: int):
     K = _f64(K)
     B, Hq, n, d = Q.shape
     Hkv = K.shape[1]
-    assert n % segment_size == 0 and n % block_size == 0
-    n1, n2 = n // segment_size, n // block_size
-    Qr = Q.reshape(B, Hq, n1, segment_size, d)
-    Kr = K.reshape(B, Hkv, n2, block_size, d)
-    return Qr.max(axis=3), Qr.min(axis=3), Kr.max(axis=3), Kr.min(axis=3)
+    def grouped(X, size):
+        """max / min over consecutive groups of `size` tokens; the last group may be shorter."""
+        groups = -(-n // size)
+        mx = np.stack([X[:, :, i * size:(i + 1) * size].max(axis=2) for i in range(groups)], axis=2)
+        mn = np.stack([X[:, :, i * size:(i + 1) * size].min(axis=2) for i in range(groups)], axis=2)
+        return mx, mn
+
+    Qmax, Qmin = grouped(Q, segment_size)
+    Kmax, Kmin = grouped(K, block_size)
+    return Qmax, Qmin, Kmax, Kmin
 
 
 def logits(Qrep: np.ndarray, Krep: np.ndarray, est_scale: float = 1.0) -> np.ndarray:

@@ -9,7 +9,9 @@ future block ever is; cnt = min(k, (j+1)*r); consistent permutation of the past 
 Readings: the r = seg/blk blocks that overlap the segment are always selected and count
 against the budget of k = B/blk blocks; the other k - r slots go to the strictly past
 blocks with the largest score, ties to the larger block index; segments that see fewer
-than k blocks take all of them (cnt < k, list padded with -1); lists are ascending.
+than k blocks take all of them (cnt < k, list padded with -1); lists are ascending.  With a
+sequence length that is not a multiple of the segment size the last segment overlaps fewer than r
+blocks and the slots it does not need go to past blocks.
 """
 from __future__ import annotations
 
@@ -22,15 +24,15 @@ def select(S: np.ndarray, segment_size: int, block_size: int, budget_blocks: int
     B, H, n1, n2 = S.shape
     r = segment_size // block_size
     k = budget_blocks
-    assert segment_size % block_size == 0 and r <= k <= n2
+    assert segment_size % block_size == 0 and r <= k
     idx = np.full((B, H, n1, k), -1, dtype=np.int32)
     cnt = np.zeros((B, H, n1), dtype=np.int32)
-    m = k - r
     for b in range(B):
         for h in range(H):
             for j in range(n1):
                 past = j * r                               # blocks strictly before the segment
-                diag = list(range(j * r, (j + 1) * r))     # blocks overlapping the segment
+                diag = list(range(j * r, min(n2, (j + 1) * r)))   # blocks overlapping the segment (fewer in a short last one)
+                m = k - len(diag)
                 if past <= m:
                     chosen = list(range(past))
                 else:

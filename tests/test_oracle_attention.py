@@ -52,11 +52,10 @@ def test_full_budget_equals_dense():
     np.testing.assert_allclose(ls, ld, rtol=1e-13)
 
 
-@pytest.mark.parametrize("seg,blk,k", [(16, 4, 6), (8, 8, 2), (12, 3, 5)])
-def test_sparse_against_mask_matrix_brute_force(seg, blk, k):
-    n = 96
+@pytest.mark.parametrize("seg,blk,k,n", [(16, 4, 6, 96), (8, 8, 2, 96), (12, 3, 5, 96), (16, 4, 6, 90), (12, 3, 5, 67)])
+def test_sparse_against_mask_matrix_brute_force(seg, blk, k, n):
     Q, K, V = qkv(n=n, seed=3)
-    n1, n2 = n // seg, n // blk
+    n1, n2 = -(-n // seg), -(-n // blk)
     S = np.random.default_rng(9).standard_normal((1, 4, n1, n2))
     idx, cnt = select(S, seg, blk, k)
     O, lse = A.sparse_attention(Q, K, V, idx, cnt, seg, blk, 0.4)
@@ -65,7 +64,7 @@ def test_sparse_against_mask_matrix_brute_force(seg, blk, k):
         for t in range(n):
             j = t // seg
             for b in idx[0, h, j, :cnt[0, h, j]]:
-                for u in range(b * blk, (b + 1) * blk):
+                for u in range(b * blk, min(n, (b + 1) * blk)):
                     allowed[t, u] = u <= t
         o2, l2 = numpy_masked_attention(Q[0, h], K[0, h // 2], V[0, h // 2], allowed, 0.4)
         np.testing.assert_allclose(O[0, h], o2, rtol=1e-12, atol=1e-14)

@@ -32,6 +32,14 @@ def test_summaries_against_token_loop():
     assert (Kr <= Kmax[:, :, :, None]).all() and (Kr >= Kmin[:, :, :, None]).all()
 
 
+def test_summaries_with_a_short_last_group():
+    Q, K = rand((1, 1, 11, 2), 20), rand((1, 1, 11, 2), 21)
+    Qmax, Qmin, Kmax, Kmin = E.summaries(Q, K, 4, 2)
+    assert Qmax.shape == (1, 1, 3, 2) and Kmax.shape == (1, 1, 6, 2)
+    assert Qmax[0, 0, 2, 1] == max(Q[0, 0, t, 1] for t in (8, 9, 10)) and Qmin[0, 0, 2, 0] == min(Q[0, 0, t, 0] for t in (8, 9, 10))
+    assert Kmax[0, 0, 5, 0] == K[0, 0, 10, 0] == Kmin[0, 0, 5, 0]
+
+
 def test_hand_worked_example():
     """n=4, d=2, seg=2, blk=1; summaries and logits below were worked out by hand."""
     Q = np.array([[1, -1], [2, 0], [0, 3], [-1, 1]], dtype=np.float64)[None, None]
@@ -72,11 +80,11 @@ def _algorithm1_probability_domain(Q, K, seg, blk, alpha, Sprev, est_scale):
     """Lines 3-14 of Algorithm 1 on probabilities in long double, loops only (one head)."""
     ld = np.longdouble
     n, d = Q.shape
-    n1, n2 = n // seg, n // blk
-    qmax = [[max(Q[j * seg + t][c] for t in range(seg)) for c in range(d)] for j in range(n1)]
-    qmin = [[min(Q[j * seg + t][c] for t in range(seg)) for c in range(d)] for j in range(n1)]
-    kmax = [[max(K[b * blk + t][c] for t in range(blk)) for c in range(d)] for b in range(n2)]
-    kmin = [[min(K[b * blk + t][c] for t in range(blk)) for c in range(d)] for b in range(n2)]
+    n1, n2 = -(-n // seg), -(-n // blk)          # a shorter last segment / block when n is not a multiple
+    qmax = [[max(Q[t][c] for t in range(j * seg, min(n, (j + 1) * seg))) for c in range(d)] for j in range(n1)]
+    qmin = [[min(Q[t][c] for t in range(j * seg, min(n, (j + 1) * seg))) for c in range(d)] for j in range(n1)]
+    kmax = [[max(K[u][c] for u in range(b * blk, min(n, (b + 1) * blk))) for c in range(d)] for b in range(n2)]
+    kmin = [[min(K[u][c] for u in range(b * blk, min(n, (b + 1) * blk))) for c in range(d)] for b in range(n2)]
 
     def smap(qr, kr):
         out = np.zeros((n1, n2), dtype=ld)
@@ -98,9 +106,9 @@ def _algorithm1_probability_domain(Q, K, seg, blk, alpha, Sprev, est_scale):
     return S
 
 
-@pytest.mark.parametrize("seg,blk", [(4, 2), (6, 3), (4, 4), (8, 2)])
-def test_log_domain_equals_probability_domain(seg, blk):
-    n, d = 24, 4
+@pytest.mark.parametrize("seg,blk,n", [(4, 2, 24), (6, 3, 24), (4, 4, 24), (8, 2, 24), (8, 2, 21), (6, 3, 19)])
+def test_log_domain_equals_probability_domain(seg, blk, n):
+    d = 4
     Q, K = 0.8 * rand((1, 1, n, d), 4 + seg), 0.8 * rand((1, 1, n, d), 5 + blk)
     S0 = _algorithm1_probability_domain(Q[0, 0], K[0, 0], seg, blk, 1.0, None, 1.0)
     L0 = E.estimate(Q, K, seg, blk)
@@ -110,7 +118,7 @@ def test_log_domain_equals_probability_domain(seg, blk):
     S1 = _algorithm1_probability_domain(Q1[0, 0], K1[0, 0], seg, blk, 0.25, S0, 1.0)
     L1 = E.estimate(Q1, K1, seg, blk, alpha=0.25, S_prev=L0)
     np.testing.assert_allclose(np.exp(L1[0, 0]), S1.astype(np.float64), rtol=1e-12, atol=0)
-    assert np.array_equal(np.isneginf(L1[0, 0]), E.causal_block_mask(n // seg, n // blk, seg, blk))
+    assert np.array_equal(np.isneginf(L1[0, 0]), E.causal_block_mask(-(-n // seg), -(-n // blk), seg, blk))
 
 
 def test_score_invariants():

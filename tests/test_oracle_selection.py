@@ -64,3 +64,20 @@ def test_future_scores_are_ignored_even_if_huge():
     for j in range(n1):
         S2[0, :, j, (j + 1) * r:] = 1e9
     assert np.array_equal(select(S, seg, blk, k)[0], select(S2, seg, blk, k)[0])
+
+
+@pytest.mark.parametrize("n,seg,blk,k", [(90, 8, 2, 6), (50, 16, 4, 5), (7, 8, 2, 4)])
+def test_short_last_segment(n, seg, blk, k):
+    """n not a multiple of the segment: the last segment overlaps fewer than r blocks and its spare
+    slots go to past blocks; a budget larger than the number of blocks selects everything."""
+    n1, n2, r = -(-n // seg), -(-n // blk), seg // blk
+    S = scores(n1, n2, 11, ties=True)
+    idx, cnt = select(S, seg, blk, k)
+    for h in range(2):
+        for j in range(n1):
+            past = list(range(j * r))
+            diag = list(range(j * r, min(n2, (j + 1) * r)))
+            ranked = sorted(past, key=lambda b: (S[0, h, j, b], b), reverse=True)
+            want = sorted(ranked[:k - len(diag)] + diag)
+            assert idx[0, h, j, :cnt[0, h, j]].tolist() == want
+            assert cnt[0, h, j] == min(k, len(past) + len(diag))
