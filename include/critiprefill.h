@@ -20,11 +20,12 @@
  *     [batch, n_kv_heads, seq_len, head_dim]; the three outer strides are given in ELEMENTS
  *     in cp_params, head_dim is contiguous.  Base pointers must be 16-byte aligned and the
  *     strides multiples of 8 elements (bf16, fp16) / 4 elements (fp32).
- *   - Notation: n1 = seq_len / segment_size, n2 = seq_len / block_size,
+ *   - Notation: n1 = ceil(seq_len / segment_size), n2 = ceil(seq_len / block_size) (the paper writes
+ *     exact divisions; a remainder leaves a shorter last segment / block),
  *     r = segment_size / block_size (blocks that overlap a segment), k = budget_blocks,
  *     g = n_q_heads / n_kv_heads; query head h uses KV head h / g.
- *   - Requirements (else CP_ERR_SHAPE): seq_len % segment_size == 0,
- *     segment_size % block_size == 0, n_q_heads % n_kv_heads == 0, r <= k <= n2.
+ *   - Requirements (else CP_ERR_SHAPE): segment_size % block_size == 0,
+ *     n_q_heads % n_kv_heads == 0, k >= r (a budget beyond the visible blocks selects them all).
  *   - Supported (else CP_ERR_UNSUPPORTED): head_dim 64 or 128; n2 <= 8192 for estimate and select;
  *     the tensor-core attention path needs bf16 or fp16, head_dim 128, segment_size % 128 == 0 and
  *     block_size in {32, 64, 128}; everything else runs on a plain SIMT kernel.
@@ -121,11 +122,12 @@ size_t critiprefill_static_scratch_bytes(void);
 
 /* Algorithm 2, line 8: I_j = argtop_k(S[j], k) with the diagonal blocks always kept.
  *   S    in   device, [B,Hq,n1,n2] fp64 (as written by critiprefill_estimate)
- *   idx  out  device, [B,Hq,n1,k] int32: ascending block indices; the r blocks overlapping
- *             segment j ([j*r,(j+1)*r)) are always present and count against k; the other
- *             k-r entries are the strictly-past blocks with the largest S[j,b], ties to the
- *             larger b; entries beyond cnt are -1
- *   cnt  out  device, [B,Hq,n1] int32 = min(k, (j+1)*r)
+ *   idx  out  device, [B,Hq,n1,k] int32: ascending block indices; the r_j blocks overlapping
+ *             segment j ([j*r, min(n2,(j+1)*r)); r_j = r except in a short last segment) are
+ *             always present and count against k; the other k-r_j entries are the
+ *             strictly-past blocks with the largest S[j,b], ties to the larger b; entries
+ *             beyond cnt are -1
+ *   cnt  out  device, [B,Hq,n1] int32 = min(k, number of blocks visible to segment j)
  * Exact (comparisons only). */
 int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws,
                         size_t ws_bytes, void* cuda_stream);
@@ -135,8 +137,8 @@ int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32
  *   U_t  = { u <= t : floor(u/block_size) in idx[b,h,j,0:cnt] },  j = floor(t/segment_size).
  *   Q, K, V   in   device
  *   idx, cnt  in   device, as produced by critiprefill_select.  Contract per list: ascending,
- *                  unique, r <= cnt <= k, and its last r entries are exactly the diagonal
- *                  blocks j*r .. (j+1)*r-1.  A list that breaks it sets CP_ERR_BOUNDS in the
+ *                  unique, r_j <= cnt <= k, and its last r_j entries are exactly the diagonal
+ *                  blocks j*r .. min(n2,(j+1)*r)-1.  A list that breaks it sets CP_ERR_BOUNDS in the
  *                  status block and its segment's rows of O are not written.
  *   O         out  device, same dtype and layout family as Q (o_stride)
  *   lse       out  device, nullable, [B,Hq,n] fp32: ln sum_{u in U_t} exp(sm_scale*q_t.k_u)

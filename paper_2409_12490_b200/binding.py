@@ -127,11 +127,11 @@ class Problem:
 
     @property
     def n1(self):
-        return self.seq_len // self.segment_size
+        return -(-self.seq_len // self.segment_size)
 
     @property
     def n2(self):
-        return self.seq_len // self.block_size
+        return -(-self.seq_len // self.block_size)
 
     def _contig(self, heads):
         n, d = self.seq_len, self.head_dim

@@ -31,11 +31,11 @@ class Config:
 
     @property
     def n1(self) -> int:
-        return self.seq_len // self.segment_size
+        return -(-self.seq_len // self.segment_size)
 
     @property
     def n2(self) -> int:
-        return self.seq_len // self.block_size
+        return -(-self.seq_len // self.block_size)
 
     @property
     def r(self) -> int:

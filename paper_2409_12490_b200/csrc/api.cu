@@ -12,9 +12,9 @@ int validate(const cp_params* p, Dims* out) {
     return CP_ERR_SHAPE;
   if (p->dtype != CP_BF16 && p->dtype != CP_F32 && p->dtype != CP_F16) return CP_ERR_UNSUPPORTED;
   if (p->n_q_heads % p->n_kv_heads) return CP_ERR_SHAPE;
-  if (p->seq_len % p->segment_size || p->segment_size % p->block_size) return CP_ERR_SHAPE;
+  if (p->segment_size % p->block_size) return CP_ERR_SHAPE;
   Dims m = make_dims(*p);
-  if (m.k < m.r || m.k > m.n2) return CP_ERR_SHAPE;
+  if (m.k < m.r) return CP_ERR_SHAPE;
   if (m.d != 64 && m.d != 128) return CP_ERR_UNSUPPORTED;
   const int64_t align = 16 / m.es;
   const int64_t* strides[4] = {p->q_stride, p->k_stride, p->v_stride, p->o_stride};

@@ -20,13 +20,14 @@ template <> __device__ __forceinline__ float from_f32<float>(float x) { return x
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
 // The list contract: ascending, in range, last r entries are the diagonal blocks of segment j.
-__device__ __forceinline__ bool list_ok(const int32_t* list, int c, int j, int r, int k, int lane) {
+__device__ __forceinline__ bool list_ok(const int32_t* list, int c, int j, int r_full, int n2, int k, int lane) {
+  const int r = min(n2, (j + 1) * r_full) - j * r_full;   // diagonal blocks of segment j
   bool ok = (c >= r) && (c <= k);
   if (ok) {
     for (int i = lane; i < c; i += 32) {
       const int v = list[i];
-      if (i >= c - r) ok = ok && (v == j * r + (i - (c - r)));
-      else ok = ok && (v >= 0) && (v < j * r) && (i == 0 || list[i - 1] < v);
+      if (i >= c - r) ok = ok && (v == j * r_full + (i - (c - r)));
+      else ok = ok && (v >= 0) && (v < j * r_full) && (i == 0 || list[i - 1] < v);
     }
   }
   return __all_sync(0xffffffffu, ok);
@@ -48,7 +49,7 @@ attention_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T*
   const int t = int(rowid % n);
   const long long bh = rowid / n;
   const int h = int(bh % Hq), b = int(bh / Hq);
-  const int j = t / seg, n1 = n / seg;
+  const int j = t / seg, n1 = (n + seg - 1) / seg, n2 = (n + blk - 1) / blk;
   const T* q = Q + b * qsb + h * qsh + int64_t(t) * qst;
   const T* Kh = K + b * ksb + (h / g) * ksh;
   const T* Vh = V + b * vsb + (h / g) * vsh;
@@ -61,7 +62,7 @@ attention_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T*
     const long long u = bh * n1 + j;
     list = idx + u * k;
     n_ranges = cnt[u];
-    if (!list_ok(list, n_ranges, j, r, k, lane)) {
+    if (!list_ok(list, n_ranges, j, r, n2, k, lane)) {
       if (lane == 0) report(st, CP_ERR_BOUNDS, 100, b, h, j, n_ranges);
       return;
     }

@@ -63,7 +63,7 @@ struct Args {
   uint16_t* O;                  // bf16 or fp16 elements
   float* lse;
   DeviceStatus* st;
-  int B, Hq, Hkv, g, n, seg, blk, k, r, n1;
+  int B, Hq, Hkv, g, n, seg, blk, k, r, n1, n2;
   int64_t osb, osh, ost;
   float sm_scale;
   int dense;
@@ -259,19 +259,20 @@ struct Unit {
   int nA, nB;       // tiles query tile A / B consumes (nB = 0: the unit has no tile B)
   const int32_t* list;
   int seg_j;
+  int rj;           // diagonal blocks of the segment (r, fewer in a short last segment)
   int cnt;
 };
 
 // Units are ordered KV-head-major so that CTAs resident at the same time share K/V tiles in
 // L2; within a KV head the dense kernel takes the longest rows first.
 // `cnt` is the unit's list length when the caller already has it, kLoadCnt to read it from global memory.
-constexpr int kLoadCnt = -2, kBadList = -1;
+constexpr int kLoadCnt = -2, kBadList = -1, kEmptyUnit = -3;   // kEmptyUnit: no query row of the unit lies inside the sequence
 __device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
   Unit u;
   u.list = nullptr;
   u.cnt = 0;
   if (a.dense) {
-    const int ntiles = a.n / kTile;
+    const int ntiles = (a.n + kTile - 1) / kTile;
     const int np = (ntiles + 1) / 2;
     const int per_kvh = a.g * np;
     const int bkv = x / per_kvh;
@@ -282,7 +283,7 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
     u.q_tok = pair * 256;
     u.n_past = 0; u.n_past_tiles = 0; u.last_cols = kTile;
     u.c_tok = 0; u.n_cont = 2 * pair; u.d_tok = pair * 256;
-    u.seg_j = 0;
+    u.seg_j = 0; u.rj = 0;
     u.nB = (2 * pair + 1 < ntiles) ? 1 : 0;
   } else {
     const int q_tiles = a.seg / kTile;
@@ -300,11 +301,12 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
     const long long unit = ((long long)u.b * a.Hq + u.h) * a.n1 + j;
     u.list = a.idx + unit * a.k;
     u.cnt = cnt == kLoadCnt ? a.cnt[unit] : cnt;
-    u.n_past = min(max(u.cnt - a.r, 0), a.k);
+    u.rj = min(a.n2, (j + 1) * a.r) - j * a.r;
+    u.n_past = min(max(u.cnt - u.rj, 0), a.k);
     u.n_past_tiles = (u.n_past * a.blk + kTile - 1) / kTile;
     u.last_cols = u.n_past * a.blk - (u.n_past_tiles - 1) * kTile;
     u.c_tok = j * a.seg; u.n_cont = 2 * p; u.d_tok = u.q_tok;
-    u.nB = (2 * p + 1 < q_tiles) ? 1 : 0;
+    u.nB = (2 * p + 1 < q_tiles && u.q_tok + kTile < a.n) ? 1 : 0;   // tile B exists and starts inside the sequence
   }
   u.nA = u.n_past_tiles + u.n_cont + 1;       // up to and including its own diagonal tile
   u.nB = u.nB ? u.nA + 1 : 0;                 // one more diagonal tile; 0 when the segment has an odd tile count
@@ -316,7 +318,7 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
 // ascending past blocks, then exactly the r diagonal blocks of the segment.
 __device__ __forceinline__ bool unit_ok(const Args& a, const Unit& u, int lane) {
   if (a.dense) return true;
-  bool ok = (u.cnt >= a.r) && (u.cnt <= a.k);
+  bool ok = (u.cnt >= u.rj) && (u.cnt <= a.k);
   if (ok) {
     for (int i = lane; i < u.cnt; i += 32) {
       const int v = u.list[i];
@@ -347,7 +349,9 @@ __device__ __forceinline__ bool publish_unit(const Args& a, Bars* bars, uint32_t
   if (x < a.n_units) {
     *u_out = decode_unit(a, x, kLoadCnt);
     cnt = u_out->cnt;
-    if (!unit_ok(a, *u_out, lane)) {
+    if (u_out->q_tok >= a.n) {
+      cnt = kEmptyUnit;                               // a short last segment has fewer units
+    } else if (!unit_ok(a, *u_out, lane)) {
       if (lane == 0) report(a.st, CP_ERR_BOUNDS, 1, u_out->b, u_out->h, u_out->seg_j, u_out->cnt);
       cnt = kBadList;
     }
@@ -388,7 +392,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
   for (uint32_t q = 0;; ++q) {
     int x, cnt;
     if (!receive_unit(a, bars, q, lane, &x, &cnt) || x >= a.n_units || stop_requested(a, bars)) return;
-    if (cnt == kBadList) continue;
+    if (cnt == kBadList || cnt == kEmptyUnit) continue;
     const Unit u = decode_unit(a, x, cnt);
     const int my_tiles = which == 0 ? u.nA : u.nB;
     if (my_tiles == 0) continue;                        // this unit has no tile B
@@ -502,10 +506,10 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
         w.y = pack2<kF16>(__uint_as_float(ov[8 * i + 2]) * inv, __uint_as_float(ov[8 * i + 3]) * inv);
         w.z = pack2<kF16>(__uint_as_float(ov[8 * i + 4]) * inv, __uint_as_float(ov[8 * i + 5]) * inv);
         w.w = pack2<kF16>(__uint_as_float(ov[8 * i + 6]) * inv, __uint_as_float(ov[8 * i + 7]) * inv);
-        dst[i] = w;
+        if (t < a.n) dst[i] = w;                     // rows past the end of the sequence (ragged last tile) are dropped
       }
     }
-    if (a.lse != nullptr)
+    if (a.lse != nullptr && t < a.n)
       a.lse[((long long)u.b * a.Hq + u.h) * a.n + t] = m_run * a.sm_scale + __logf(l_run);
   }
 }
@@ -526,7 +530,7 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
     if (x >= a.n_units || stop_requested(a, bars)) return;
     const Unit u_cur = u;
     if (!publish_unit(a, bars, q + 1, lane, &x, &u)) return;
-    if (u_cur.cnt == kBadList) continue;
+    if (u_cur.cnt == kBadList || u_cur.cnt == kEmptyUnit) continue;
     // Q tiles: the buffer is free once every QK^T of the previous unit has completed
     if (n_units > 0 && !mbar_wait(&bars->q_empty, (n_units - 1) & 1, bars, a.st, 31)) return;
     if (lane == 0) {
@@ -601,7 +605,7 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
   for (uint32_t q = 0;; ++q) {
     int x, cnt;
     if (!receive_unit(a, bars, q, lane, &x, &cnt) || x >= a.n_units || stop_requested(a, bars)) return;
-    if (cnt == kBadList) continue;
+    if (cnt == kBadList || cnt == kEmptyUnit) continue;
     const Unit u = decode_unit(a, x, cnt);
     const int T = u.T, TA = u.nA;
     const bool hasB = u.nB > 0;
@@ -752,11 +756,11 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
   Args a;
   a.idx = idx; a.cnt = cnt; a.O = static_cast<uint16_t*>(O); a.lse = lse; a.st = st;
   a.B = m.B; a.Hq = m.Hq; a.Hkv = m.Hkv; a.g = m.g; a.n = m.n; a.seg = m.seg; a.blk = m.blk; a.k = m.k;
-  a.r = m.r; a.n1 = m.n1;
+  a.r = m.r; a.n1 = m.n1; a.n2 = m.n2;
   a.osb = p.o_stride[0]; a.osh = p.o_stride[1]; a.ost = p.o_stride[2];
   a.sm_scale = p.sm_scale; a.dense = dense ? 1 : 0;
   // a unit is two 128-row query tiles (one when a segment, or the sequence, has an odd tile count)
-  const long long units = dense ? (long long)m.B * m.Hq * ((m.n / kTile + 1) / 2)
+  const long long units = dense ? (long long)m.B * m.Hq * (((m.n + kTile - 1) / kTile + 1) / 2)
                                 : (long long)m.B * m.Hq * m.n1 * ((m.seg / kTile + 1) / 2);
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
   auto kern = f16 ? attention_sm100_kernel<true> : attention_sm100_kernel<false>;

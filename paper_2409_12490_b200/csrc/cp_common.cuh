@@ -21,7 +21,9 @@ inline Dims make_dims(const cp_params& p) {
   Dims m;
   m.B = p.batch; m.Hq = p.n_q_heads; m.Hkv = p.n_kv_heads; m.g = p.n_q_heads / p.n_kv_heads;
   m.n = p.seq_len; m.d = p.head_dim; m.seg = p.segment_size; m.blk = p.block_size;
-  m.k = p.budget_blocks; m.n1 = p.seq_len / p.segment_size; m.n2 = p.seq_len / p.block_size;
+  m.k = p.budget_blocks;
+  m.n1 = (p.seq_len + p.segment_size - 1) / p.segment_size;   // the last segment / block may be shorter
+  m.n2 = (p.seq_len + p.block_size - 1) / p.block_size;
   m.r = p.segment_size / p.block_size; m.es = p.dtype == CP_F32 ? 4 : 2;
   return m;
 }

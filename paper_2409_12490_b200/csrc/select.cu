@@ -36,11 +36,12 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
   const double* row = S + size_t(unit) * n2;
   int32_t* out = idx + size_t(unit) * k;
   const int past = j * r;
-  const int m = k - r;
+  const int rj = min(n2, past + r) - past;   // diagonal blocks of this segment (fewer in a short last segment)
+  const int m = k - rj;
 
   if (past <= m) {
     // every visible block fits in the budget
-    const int c = past + r;
+    const int c = past + rj;
     for (int i = tid; i < k; i += kThreads) out[i] = i < c ? i : -1;
     if (tid == 0) cnt[unit] = c;
     return;
@@ -48,8 +49,8 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
 
   if (m == 0) {
     // the budget holds the diagonal blocks only
-    for (int i = tid; i < r; i += kThreads) out[i] = past + i;
-    if (tid == 0) cnt[unit] = k;
+    for (int i = tid; i < k; i += kThreads) out[i] = i < rj ? past + i : -1;
+    if (tid == 0) cnt[unit] = rj;
     return;
   }
 
@@ -140,7 +141,7 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
     }
     __syncthreads();
   }
-  for (int i = tid; i < r; i += kThreads) out[m + i] = past + i;   // diagonal blocks
+  for (int i = tid; i < rj; i += kThreads) out[m + i] = past + i;   // diagonal blocks
   if (tid == 0) cnt[unit] = k;
 }
 

@@ -17,6 +17,7 @@ constexpr int kThreads = kWarps * 32;
 template <typename T> struct Vec;
 template <> struct Vec<__nv_bfloat16> {
   uint4 v;
+  static constexpr uint32_t kNegInf = 0xFF80FF80u, kPosInf = 0x7F807F80u;   // packed pairs
   __device__ static Vec load(const void* p) { Vec r; r.v = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
   __device__ void store(void* p) const { *reinterpret_cast<uint4*>(p) = v; }
   __device__ static uint32_t mx(uint32_t a, uint32_t b) {
@@ -30,6 +31,7 @@ template <> struct Vec<__nv_bfloat16> {
 };
 template <> struct Vec<__half> {
   uint4 v;
+  static constexpr uint32_t kNegInf = 0xFC00FC00u, kPosInf = 0x7C007C00u;
   __device__ static Vec load(const void* p) { Vec r; r.v = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
   __device__ void store(void* p) const { *reinterpret_cast<uint4*>(p) = v; }
   __device__ static uint32_t mx(uint32_t a, uint32_t b) {
@@ -43,6 +45,7 @@ template <> struct Vec<__half> {
 };
 template <> struct Vec<float> {
   uint4 v;
+  static constexpr uint32_t kNegInf = 0xFF800000u, kPosInf = 0x7F800000u;
   __device__ static Vec load(const void* p) { Vec r; r.v = __ldg(reinterpret_cast<const uint4*>(p)); return r; }
   __device__ void store(void* p) const { *reinterpret_cast<uint4*>(p) = v; }
   __device__ static uint32_t mx(uint32_t a, uint32_t b) { return __float_as_uint(fmaxf(__uint_as_float(a), __uint_as_float(b))); }
@@ -67,21 +70,22 @@ __device__ __forceinline__ uint4 shfl_xor4(const uint4& a, int m) {
 struct Side {            // one tensor (Q or K) and where its summaries go
   const char* base;      // element (b,h,t,0) at base + (b*sb + h*sh + t*st) * es
   int64_t sb, sh, st;    // strides in elements
-  int H, groups_per_head, G;  // heads, groups per head (n/G), rows per group
+  int H, groups_per_head, G, n;  // heads, groups per head (ceil(n/G)), rows per group (the last may be shorter), tokens
   char *omax, *omin;     // [B,H,groups,d] contiguous
   long long n_groups;    // B*H*groups_per_head
   long long cta_begin;   // first CTA of this side
   int groups_per_cta;    // kWarps (warp-owned groups) or 1 (CTA-owned group)
 };
 
-// Reduce rows [row0, row0+nrows) strided by `rstride` rows among callers; returns the lane's
-// 16-byte slice of (max, min).
+// Fold rows first+sub, first+sub+step, ... (< first+nrows) of a group into the lane's 16-byte
+// slice of (max, min).  The accumulators start at -inf / +inf, so a lane without rows is neutral.
 template <typename T, int LPR>
 __device__ __forceinline__ void scan_rows(const char* gbase, int64_t st_bytes, int first, int nrows,
                                           int step, int lane, uint4& mx, uint4& mn) {
   const int sub = lane / LPR, col = lane % LPR;
   const char* p0 = gbase + int64_t(first + sub) * st_bytes + col * 16;
-  bool init = false;
+  mx = make_uint4(Vec<T>::kNegInf, Vec<T>::kNegInf, Vec<T>::kNegInf, Vec<T>::kNegInf);
+  mn = make_uint4(Vec<T>::kPosInf, Vec<T>::kPosInf, Vec<T>::kPosInf, Vec<T>::kPosInf);
   constexpr int UNROLL = 8;
   int i = first + sub;
   const int end = first + nrows;
@@ -89,13 +93,11 @@ __device__ __forceinline__ void scan_rows(const char* gbase, int64_t st_bytes, i
     uint4 v[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) v[u] = Vec<T>::load(p0 + int64_t(i - first - sub + u * step) * st_bytes).v;
-    if (!init) { mx = v[0]; mn = v[0]; init = true; }
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) { vmax<T>(mx, v[u]); vmin<T>(mn, v[u]); }
   }
   for (; i < end; i += step) {
-    uint4 v = Vec<T>::load(p0 + int64_t(i - first - sub) * st_bytes).v;
-    if (!init) { mx = v; mn = v; init = true; }
+    const uint4 v = Vec<T>::load(p0 + int64_t(i - first - sub) * st_bytes).v;
     vmax<T>(mx, v); vmin<T>(mn, v);
   }
 }
@@ -117,8 +119,9 @@ __global__ void __launch_bounds__(kThreads) summarize_kernel(Side q, Side k, int
     const long long bh = grp / s.groups_per_head;
     const int h = int(bh % s.H), b = int(bh / s.H);
     const char* gbase = s.base + (int64_t(b) * s.sb + int64_t(h) * s.sh + int64_t(gi) * s.G * s.st) * es;
+    const int rows = min(s.G, s.n - gi * s.G);
     uint4 mx, mn;
-    scan_rows<T, LPR>(gbase, st_bytes, warp * RPW, s.G - warp * RPW, kWarps * RPW, lane, mx, mn);
+    scan_rows<T, LPR>(gbase, st_bytes, warp * RPW, rows - warp * RPW, kWarps * RPW, lane, mx, mn);
 #pragma unroll
     for (int m = LPR; m < 32; m <<= 1) { uint4 o = shfl_xor4(mx, m); vmax<T>(mx, o); o = shfl_xor4(mn, m); vmin<T>(mn, o); }
     if (lane < LPR) { red[0][warp][lane] = mx; red[1][warp][lane] = mn; }
@@ -139,19 +142,11 @@ __global__ void __launch_bounds__(kThreads) summarize_kernel(Side q, Side k, int
     const long long bh = grp / s.groups_per_head;
     const int h = int(bh % s.H), b = int(bh / s.H);
     const char* gbase = s.base + (int64_t(b) * s.sb + int64_t(h) * s.sh + int64_t(gi) * s.G * s.st) * es;
+    const int rows = min(s.G, s.n - gi * s.G);
     uint4 mx, mn;
-    if (s.G >= RPW) {
-      scan_rows<T, LPR>(gbase, st_bytes, 0, s.G, RPW, lane, mx, mn);
+    scan_rows<T, LPR>(gbase, st_bytes, 0, rows, RPW, lane, mx, mn);
 #pragma unroll
-      for (int m = LPR; m < 32; m <<= 1) { uint4 o = shfl_xor4(mx, m); vmax<T>(mx, o); o = shfl_xor4(mn, m); vmin<T>(mn, o); }
-    } else {
-      // fewer rows than the warp covers: lanes of sub-row >= G idle; fold only valid sub-rows
-      const int sub = lane / LPR, col = lane % LPR;
-      uint4 v = Vec<T>::load(gbase + int64_t(sub < s.G ? sub : 0) * st_bytes + col * 16).v;
-      mx = v; mn = v;
-#pragma unroll
-      for (int m = LPR; m < 32; m <<= 1) { uint4 o = shfl_xor4(mx, m); vmax<T>(mx, o); o = shfl_xor4(mn, m); vmin<T>(mn, o); }
-    }
+    for (int m = LPR; m < 32; m <<= 1) { uint4 o = shfl_xor4(mx, m); vmax<T>(mx, o); o = shfl_xor4(mn, m); vmin<T>(mn, o); }
     if (lane < LPR) {
       const size_t off = (size_t(grp) * d) * es + lane * 16;
       *reinterpret_cast<uint4*>(s.omax + off) = mx;
@@ -174,7 +169,7 @@ int launch_summarize(const cp_params& p, const Dims& m, const void* Q, const voi
   auto mk = [&](const void* base, const int64_t* s, int H, int G, char* omax, char* omin) {
     Side x;
     x.base = static_cast<const char*>(base); x.sb = s[0]; x.sh = s[1]; x.st = s[2];
-    x.H = H; x.G = G; x.groups_per_head = m.n / G; x.omax = omax; x.omin = omin;
+    x.H = H; x.G = G; x.n = m.n; x.groups_per_head = (m.n + G - 1) / G; x.omax = omax; x.omin = omin;
     x.n_groups = (long long)m.B * H * x.groups_per_head;
     x.groups_per_cta = G > 128 ? 1 : kWarps;
     x.cta_begin = 0;

@@ -37,7 +37,8 @@ def test_host_validation_without_gpu():
     with pytest.raises(cp.CritiPrefillError):
         cp.workspace_bytes(cp.Problem(1, 4, 3, 1024, 64, 128, 32, 8))      # Hq % Hkv
     with pytest.raises(cp.CritiPrefillError):
-        cp.workspace_bytes(cp.Problem(1, 4, 2, 1000, 64, 128, 32, 8))      # n % seg
+        cp.workspace_bytes(cp.Problem(1, 4, 2, 1024, 64, 128, 48, 8))      # seg % blk
     with pytest.raises(cp.CritiPrefillError):
         cp.workspace_bytes(cp.Problem(1, 4, 2, 1024, 64, 128, 32, 3))      # k < r
+    assert cp.workspace_bytes(cp.Problem(1, 4, 2, 1000, 64, 128, 32, 8)) > 256   # a ragged length is fine
     assert "workspace" in cp.status_string(4)

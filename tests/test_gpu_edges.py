@@ -166,3 +166,25 @@ def test_fp16_inputs_whole_path(flags):
     assert cp.device_status(ws) == 0
     O_ref, _ = oracle.dense_attention(Q, K, V, f32(1.0 / np.sqrt(cfg.head_dim)))
     assert_attention_close(Od, O_ref)
+
+
+@pytest.mark.parametrize("n,seg,blk,d,dtype", [(1000, 256, 64, 128, "bf16"), (1340, 256, 32, 128, "bf16"),
+                                               (777, 128, 128, 128, "f16"), (200, 256, 64, 128, "bf16"),
+                                               (1000, 128, 32, 64, "f32")])
+def test_sequence_lengths_that_are_not_multiples(n, seg, blk, d, dtype):
+    """A shorter last segment / block (n1 = ceil(n/seg), n2 = ceil(n/blk)): every step against the oracle,
+    plus the dense kernel, and nothing is written past the end of O."""
+    cfg = BASE.with_(seq_len=n, segment_size=seg, block_size=blk, budget_tokens=2 * seg, head_dim=d, dtype=dtype,
+                     n_q_heads=4, n_kv_heads=2)
+    Q, K, V = make_qkv(cfg)
+    tol = (1e-5, 1e-6) if dtype == "f32" else (TOL_BF16_MAX, TOL_BF16_MEAN)
+    full_path_vs_oracle(cfg, Q, K, V, tol=tol)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    guard = torch.full((1, cfg.n_q_heads, n + 8, d), 7.0, dtype=Q.dtype, device="cuda")   # canary rows behind every head
+    Od = cp.dense_attention(prob, Qd, Kd, Vd, ws, O=guard[:, :, :n])
+    assert cp.device_status(ws) == 0
+    assert (guard[:, :, n:] == 7.0).all()
+    O_ref, _ = oracle.dense_attention(Q, K, V, f32(1.0 / np.sqrt(d)))
+    assert_attention_close(Od, O_ref, *tol)

@@ -176,7 +176,7 @@ def test_host_side_argument_errors():
     with pytest.raises(cp.CritiPrefillError) as e:
         cp.estimate(prob, Q, K, ws[:1024])
     assert e.value.status == 4
-    bad = cp.Problem.from_config(cfg.with_(segment_size=192))
+    bad = cp.Problem.from_config(cfg.with_(segment_size=200))        # not a multiple of the block size
     with pytest.raises(cp.CritiPrefillError) as e:
         cp.workspace_bytes(bad)
     assert e.value.status == 2
