@@ -30,9 +30,11 @@ from paper_2409_12490_b200.sharding import RankInfo, aggregate_time_metric, laye
 
 METRIC = "128K prefill-attention ms (estimate+select+sparse attention, one layer)"
 # DRAM bytes (read + write) per launch of the sparse attention kernel, from the ncu captures
-# summarised in profiles/attention_sm100_kernel_C4_dram.md (C4, full size) and
+# summarised in profiles/attention_sm100_kernel_C4_counters.md (C4, full size) and
 # profiles/attention_sm100_kernel_C3.md; None for workloads without a capture.
 ATTN_TRAFFIC_BYTES = {"C4": 2.80e9, "C3": 0.635e9}
+# sm__pipe_tensor_cycles_active (% of peak, elapsed) of the same kernel from the same captures
+ATTN_TENSOR_PIPE_PCT = {"C4": 56.7, "C3": 46.2}
 
 
 def load_peaks():
@@ -366,6 +368,7 @@ def run_ours(args, cfg):
                 "frac": achieved / peaks["bf16_tflops"], "peak_source": f"{peaks['source']} (burst)",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
                 "flops_per_launch": fl["executed"], "traffic": ATTN_TRAFFIC_BYTES.get(cfg.name),
+                "tensor_pipe_active_pct_ncu": ATTN_TENSOR_PIPE_PCT.get(cfg.name),
                 "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, ncu)"}
     summary_bytes = (dQ.numel() + dK.numel()) * dQ.element_size()
     out = {
