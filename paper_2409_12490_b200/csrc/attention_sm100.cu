@@ -36,7 +36,7 @@ constexpr int kSmemBar = kSmemKV + kSlots * kTileBytes;
 constexpr int kSmemTotal = kSmemBar + 256 + 1024;   // + barrier block + slack to align the tiles to 1024 bytes
 constexpr float kRescaleThreshold = 8.0f;           // in log2 units
 #ifndef CP_EMUL_EVERY
-#define CP_EMUL_EVERY 4
+#define CP_EMUL_EVERY 8
 #endif
 constexpr int kEmulEvery = CP_EMUL_EVERY;           // 0: all exponentials on the MUFU; n: every n-th pair on the FMA pipes
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
