@@ -11,6 +11,8 @@ causality; GQA = MHA with replicated KV heads; a single-block list in closed for
 
 Readings: softmax runs over the selected keys only (Algorithm 2, line 10, as written), with
 token-level causality u <= t applied inside the selected blocks (the paper's decoder setting).
+The arithmetic is pinned (tests above); the causal reading inside Algorithm 2 is parity unpinned against
+the authors' code.
 """
 from __future__ import annotations
 

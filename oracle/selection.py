@@ -12,6 +12,7 @@ blocks with the largest score, ties to the larger block index; segments that see
 than k blocks take all of them (cnt < k, list padded with -1); lists are ascending.  With a
 sequence length that is not a multiple of the segment size the last segment overlaps fewer than r
 blocks and the slots it does not need go to past blocks.
+The selection itself is pinned (tests above); which reading the authors' code takes is parity unpinned.
 """
 from __future__ import annotations
 

@@ -188,3 +188,39 @@ def test_sequence_lengths_that_are_not_multiples(n, seg, blk, d, dtype):
     assert (guard[:, :, n:] == 7.0).all()
     O_ref, _ = oracle.dense_attention(Q, K, V, f32(1.0 / np.sqrt(d)))
     assert_attention_close(Od, O_ref, *tol)
+
+
+def test_repeated_runs_are_bit_identical_and_stay_inside_their_buffers():
+    """No atomics touch the outputs, so two runs must agree bit for bit; every output buffer sits
+    inside a poisoned allocation whose padding must come back untouched."""
+    cfg = CONFIGS["C2"].with_(name="det", seq_len=4096, n_q_heads=8, n_kv_heads=2, segment_size=512, block_size=64,
+                              budget_tokens=1024, n_clusters=16)
+    Q, K, V = make_qkv(cfg)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    pad = 64
+
+    def padded(shape, dtype, fill):
+        flat = torch.full((int(np.prod(shape)) + 2 * pad,), fill, dtype=dtype, device="cuda")
+        return flat, flat[pad:-pad].view(shape)
+
+    outs = []
+    for _ in range(2):
+        S_raw, S = padded((1, cfg.n_q_heads, cfg.n1, cfg.n2), torch.float64, float("nan"))
+        i_raw, idx = padded((1, cfg.n_q_heads, cfg.n1, cfg.budget_blocks), torch.int32, -7)
+        c_raw, cnt = padded((1, cfg.n_q_heads, cfg.n1), torch.int32, -7)
+        O_raw, O = padded(tuple(Qd.shape), torch.bfloat16, float("nan"))
+        l_raw, lse = padded((1, cfg.n_q_heads, cfg.seq_len), torch.float32, float("nan"))
+        cp.estimate(prob, Qd, Kd, ws, S_out=S)
+        cp.select(prob, S, ws, idx=idx, cnt=cnt)
+        cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws, O=O, lse=lse)
+        assert cp.device_status(ws) == 0
+        for raw in (S_raw, O_raw, l_raw):
+            assert torch.isnan(raw[:pad]).all() and torch.isnan(raw[-pad:]).all()
+        for raw in (i_raw, c_raw):
+            assert (raw[:pad] == -7).all() and (raw[-pad:] == -7).all()
+        assert not torch.isnan(O.float()).any() and not torch.isnan(lse).any()
+        outs.append((S.clone(), idx.clone(), cnt.clone(), O.clone(), lse.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
