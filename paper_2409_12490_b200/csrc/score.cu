@@ -27,12 +27,13 @@ __device__ __forceinline__ double logaddexp(double a, double b) {
   const double hi = fmax(a, b), lo = fmin(a, b);
   const double d = lo - hi;                 // <= 0, or NaN when both are -inf
   if (!(d > -50.0)) return hi;
-  return hi + log1p(exp(d));
+  return hi + log(1.0 + exp(d));            // absolute error ~2e-16, as good as log1p once it is added to hi
 }
 
-// Shared memory: logits lg[U][4][nb] for the nb key blocks this CTA owns.  When the 4*U*n2 logits
-// of a row group do not fit one CTA's shared memory, CL CTAs of a thread-block cluster split the
-// key blocks and merge their per-row (max, sum) pairs through distributed shared memory.
+// Shared memory: logits lg[U][4][nb] (fp64) for the nb key blocks this CTA owns, plus an fp32 copy that
+// the log-sum-exp uses as a filter.  When the 4*U*n2 logits of a row group do not fit one CTA's shared
+// memory, CL CTAs of a thread-block cluster split the key blocks and merge their per-row (max, sum)
+// pairs through distributed shared memory.
 template <typename T, int D, int U>
 __global__ void __launch_bounds__(kThreads)
 score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __restrict__ Kmax,
@@ -41,6 +42,7 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
              double ln_1m_alpha, int fuse, int mask_first, int CL, int nb) {
   extern __shared__ double smem[];
   double* lg = smem;                                // [U][4][nb]
+  float* lf = reinterpret_cast<float*>(smem + 4 * U * nb);   // the same logits rounded to fp32: a cheap filter for the log-sum-exp
   __shared__ double stat[4 * U];
   __shared__ double2 part[4 * U];                   // this CTA's (max, sum exp) per logit row
 
@@ -66,74 +68,130 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   const T* kmx_base = Kmax + size_t(kvh) * n2 * D;
   const T* kmn_base = Kmin + size_t(kvh) * n2 * D;
 
-  // The 8 x n2 x D logit products run on the fp64 tensor-core path (mma.m8n8k4): the 8 rows of
-  // A are (head u, representative) = (u0 max, u0 min, u1 max, ...); B columns are key blocks.
-  // Lane l supplies A[l/4][l%4] and B[l%4][l/4] per k-step and owns C[l/4][2(l%4)+{0,1}].
-  // The channel order inside the dot product is free, so lane-in-quad q takes the D/4
-  // contiguous channels [q*D/4, (q+1)*D/4): one contiguous slice of a summary row per lane.
-  constexpr int KS = D / 4;                 // k-steps
-  constexpr int VE = 16 / sizeof(T);        // elements per 16-byte load
-  constexpr int NV = KS / VE;               // 16-byte loads per lane per row
-  const int quad = lane & 3, grp = lane >> 2;
-  double afrag[KS];
-  {
-    const int u = grp >> 1, rep = grp & 1;
-    const T* src = (rep == 0 ? Qmax : Qmin) + (u < U ? unit_of(u) : unit_of(0)) * D + quad * KS;
-#pragma unroll
-    for (int ks = 0; ks < KS; ++ks) afrag[ks] = u < U ? to_f64(src[ks]) : 0.0;
+  // The 8 x n2 x D logit products run on the fp64 tensor cores as mma.m16n8k16 with the key blocks on the
+  // M side: per warp tile, A = 16 key blocks x 16 channels (streamed from the summaries, widened to fp64),
+  // B = 16 channels x 8 columns, the columns being (head u, representative) = (u0 max, u0 min, u1 max, ...),
+  // C = 16 blocks x 8 columns.  Lane (grp = lane/4, tig = lane%4) supplies A[grp | grp+8][c*4+tig],
+  // B[i*4+tig][grp] and owns C[grp | grp+8][2*tig + {0,1}].  The channel order inside a dot product is
+  // free, so lane tig takes the D/4 contiguous channels [tig*D/4, (tig+1)*D/4) of a summary row, four of
+  // them per MMA: 16-byte loads, and each key value is converted once per CTA.
+  constexpr int KS = D / 4;                 // channels per lane slice
+  constexpr int CE = 16 / sizeof(T);        // elements per 16-byte load
+  constexpr int NCH = KS / CE;              // loads per slice
+  constexpr int SPC = CE / 4;               // MMA k-steps per load
+  constexpr int QS = D + 2;                 // row stride of qs in doubles (odd number of 16-byte units: conflict-free)
+  __shared__ __align__(16) double qs[8 * QS];   // B operand, row = column index n, laid out [k-step][tig][4 channels]
+  const int tig = lane & 3, grp = lane >> 2;
+  for (int e = tid; e < 8 * D; e += kThreads) {
+    const int n = e / D, ch = e % D;        // column n = (head n/2, representative n%2); channel ch
+    const int u = n >> 1, rep = n & 1;
+    const int tq = ch / KS, within = ch % KS;                         // owner lane-in-quad, position in its slice
+    const double v = u < U ? to_f64(((rep == 0 ? Qmax : Qmin) + unit_of(u) * D)[ch]) : 0.0;
+    qs[n * QS + ((within >> 2) * 4 + tq) * 4 + (within & 3)] = v;
   }
-  const int n_tiles = (nloc + 7) / 8;
+  __syncthreads();
+  const int n_tiles = (nloc + 15) / 16;
   for (int t = warp; t < n_tiles; t += kWarps) {
-    const int bblk = b_lo + min(t * 8 + grp, nloc - 1);  // this lane's B column (clamped in a ragged last tile)
-    const uint4* pmx = reinterpret_cast<const uint4*>(kmx_base + size_t(bblk) * D + quad * KS);
-    const uint4* pmn = reinterpret_cast<const uint4*>(kmn_base + size_t(bblk) * D + quad * KS);
-    uint4 vx[NV], vn[NV];
+    // this lane's two A rows (clamped in a ragged last tile), for the max and the min summaries
+    const int blk0 = b_lo + min(t * 16 + grp, nloc - 1), blk1 = b_lo + min(t * 16 + grp + 8, nloc - 1);
+    const uint4* src[4] = {reinterpret_cast<const uint4*>(kmx_base + size_t(blk0) * D + tig * KS),
+                           reinterpret_cast<const uint4*>(kmx_base + size_t(blk1) * D + tig * KS),
+                           reinterpret_cast<const uint4*>(kmn_base + size_t(blk0) * D + tig * KS),
+                           reinterpret_cast<const uint4*>(kmn_base + size_t(blk1) * D + tig * KS)};
+    double cx[4] = {0.0, 0.0, 0.0, 0.0}, cn[4] = {0.0, 0.0, 0.0, 0.0};
+    uint4 cur[4], nxt[4];
 #pragma unroll
-    for (int v = 0; v < NV; ++v) { vx[v] = __ldg(pmx + v); vn[v] = __ldg(pmn + v); }
-    double cx0 = 0.0, cx1 = 0.0, cn0 = 0.0, cn1 = 0.0;
+    for (int i = 0; i < 4; ++i) cur[i] = __ldg(src[i]);
 #pragma unroll
-    for (int v = 0; v < NV; ++v) {
-      const T* ka = reinterpret_cast<const T*>(&vx[v]);
-      const T* kc = reinterpret_cast<const T*>(&vn[v]);
+    for (int ch = 0; ch < NCH; ++ch) {
+      if (ch + 1 < NCH) {
 #pragma unroll
-      for (int e = 0; e < VE; ++e) {
-        const double a = afrag[v * VE + e];
-        const double bx = to_f64(ka[e]), bn = to_f64(kc[e]);
-        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                     : "+d"(cx0), "+d"(cx1) : "d"(a), "d"(bx));
-        asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                     : "+d"(cn0), "+d"(cn1) : "d"(a), "d"(bn));
+        for (int i = 0; i < 4; ++i) nxt[i] = __ldg(src[i] + ch + 1);
+      }
+#pragma unroll
+      for (int sp = 0; sp < SPC; ++sp) {
+        const int step = ch * SPC + sp;
+        double ax[8], an[8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          ax[2 * c] = to_f64(reinterpret_cast<const T*>(&cur[0])[sp * 4 + c]);
+          ax[2 * c + 1] = to_f64(reinterpret_cast<const T*>(&cur[1])[sp * 4 + c]);
+          an[2 * c] = to_f64(reinterpret_cast<const T*>(&cur[2])[sp * 4 + c]);
+          an[2 * c + 1] = to_f64(reinterpret_cast<const T*>(&cur[3])[sp * 4 + c]);
+        }
+        const double2 b01 = *reinterpret_cast<const double2*>(&qs[grp * QS + (step * 4 + tig) * 4]);
+        const double2 b23 = *reinterpret_cast<const double2*>(&qs[grp * QS + (step * 4 + tig) * 4 + 2]);
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f64.f64.f64.f64 {%0,%1,%2,%3}, {%4,%5,%6,%7,%8,%9,%10,%11}, "
+            "{%12,%13,%14,%15}, {%0,%1,%2,%3};"
+            : "+d"(cx[0]), "+d"(cx[1]), "+d"(cx[2]), "+d"(cx[3])
+            : "d"(ax[0]), "d"(ax[1]), "d"(ax[2]), "d"(ax[3]), "d"(ax[4]), "d"(ax[5]), "d"(ax[6]), "d"(ax[7]),
+              "d"(b01.x), "d"(b01.y), "d"(b23.x), "d"(b23.y));
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f64.f64.f64.f64 {%0,%1,%2,%3}, {%4,%5,%6,%7,%8,%9,%10,%11}, "
+            "{%12,%13,%14,%15}, {%0,%1,%2,%3};"
+            : "+d"(cn[0]), "+d"(cn[1]), "+d"(cn[2]), "+d"(cn[3])
+            : "d"(an[0]), "d"(an[1]), "d"(an[2]), "d"(an[3]), "d"(an[4]), "d"(an[5]), "d"(an[6]), "d"(an[7]),
+              "d"(b01.x), "d"(b01.y), "d"(b23.x), "d"(b23.y));
+      }
+      if (ch + 1 < NCH) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
       }
     }
-    // C rows: grp = (u, rep); rep 0 (Qmax): cx = l1, cn = l2; rep 1 (Qmin): cx = l3, cn = l4
-    const int u = grp >> 1, rep = grp & 1;
-    if (u < U) {
+    // C[i]: block grp + 8*(i/2), column 2*tig + (i%2) = (head tig, representative i%2);
+    // representative 0 (Qmax): cx = l1, cn = l2; representative 1 (Qmin): cx = l3, cn = l4
+    if (tig < U) {
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        const int lb = t * 8 + quad * 2 + i;           // local block index
+      for (int i = 0; i < 4; ++i) {
+        const int lb = t * 16 + grp + (i >> 1) * 8;      // local block index
+        const int rep = i & 1;
         if (lb < nloc) {
           const bool hide = mask_first && b_lo + lb >= visible;
-          lg[(u * 4 + rep * 2 + 0) * nb + lb] = hide ? -CUDART_INF : (i ? cx1 : cx0) * est_scale;
-          lg[(u * 4 + rep * 2 + 1) * nb + lb] = hide ? -CUDART_INF : (i ? cn1 : cn0) * est_scale;
+          const double vx = hide ? -CUDART_INF : cx[i] * est_scale, vn = hide ? -CUDART_INF : cn[i] * est_scale;
+          lg[(tig * 4 + rep * 2 + 0) * nb + lb] = vx;
+          lg[(tig * 4 + rep * 2 + 1) * nb + lb] = vn;
+          lf[(tig * 4 + rep * 2 + 0) * nb + lb] = float(vx);
+          lf[(tig * 4 + rep * 2 + 1) * nb + lb] = float(vn);
         }
       }
     }
   }
   __syncthreads();
 
-  // log-sum-exp of each of the 4U logit rows (softmax over blocks, lines 9-10): a warp owns a
-  // row, so only shuffles are needed; terms more than e^-50 below the maximum are skipped
+  // log-sum-exp of each of the 4U logit rows (softmax over blocks, lines 9-10): a warp owns a row, so only
+  // shuffles are needed.  Terms more than e^-50 below the row maximum cannot change the rounded sum and
+  // are skipped.  Only a few percent of a row survive that test, scattered over the lanes, so the row is
+  // first scanned in fp32 and the candidates -- fp32 value within 50 + a rounding margin of the fp32
+  // maximum, which always includes the true maximum and every term that counts -- are compacted into a
+  // dense index list (in place, over the fp32 row); the fp64 maximum and the exponentials then run on full warps.
 #pragma unroll 1
   for (int rI = warp; rI < 4 * U; rI += kWarps) {
     const double* rowp = lg + rI * nb;
+    float* rowf = lf + rI * nb;
+    float mf = -CUDART_INF_F;
+#pragma unroll 4
+    for (int lb = lane; lb < nloc; lb += 32) mf = fmaxf(mf, rowf[lb]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mf = fmaxf(mf, __shfl_xor_sync(0xffffffffu, mf, o));
+    const float thr = mf - (51.0f + fabsf(mf) * 1e-6f);     // -inf when the whole (local) row is masked: no candidates
+    int* cand = reinterpret_cast<int*>(rowf);                // entry i is written after element i has been read
+    int ncand = 0;
+    for (int base = 0; base < nloc; base += 32) {
+      const int lb = base + lane;
+      const bool c = lb < nloc && rowf[lb] > thr;
+      const unsigned ballot = __ballot_sync(0xffffffffu, c);
+      if (c) cand[ncand + __popc(ballot & ((1u << lane) - 1u))] = lb;
+      ncand += __popc(ballot);
+    }
+    __syncwarp();
     double m = -CUDART_INF;
-    for (int lb = lane; lb < nloc; lb += 32) m = fmax(m, rowp[lb]);
+    for (int i = lane; i < ncand; i += 32) m = fmax(m, rowp[cand[i]]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
     double sum = 0.0;
-#pragma unroll 4
-    for (int lb = lane; lb < nloc; lb += 32) {
-      const double d = rowp[lb] - m;
+    for (int i = lane; i < ncand; i += 32) {
+      const double d = rowp[cand[i]] - m;
       if (d > -50.0) sum += exp(d);
     }
 #pragma unroll
@@ -145,17 +203,19 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     cluster.sync();                                   // every CTA's partials are in place
-    if (tid < 4 * U) {
-      double M = -CUDART_INF;
-      for (int r = 0; r < CL; ++r) M = fmax(M, cluster.map_shared_rank(part, r)[tid].x);
-      double Ssum = 0.0;
-      for (int r = 0; r < CL; ++r) {
-        const double2 pr = cluster.map_shared_rank(part, r)[tid];
-        if (pr.y > 0.0) Ssum += pr.y * exp(pr.x - M);
-      }
-      stat[tid] = M + log(Ssum);
+    // thread (row, r) fetches rank r's pair of that row; the CL lanes of a row are adjacent, so the merge is shuffles
+    if (warp * 32 < 4 * U * CL) {                     // whole warps take part in the shuffles
+      const bool act = tid < 4 * U * CL;
+      const int row = act ? tid / CL : 0, r = tid % CL;
+      const double2 pr = cluster.map_shared_rank(part, r)[row];
+      double M = pr.x;
+      for (int o = CL >> 1; o > 0; o >>= 1) M = fmax(M, __shfl_xor_sync(0xffffffffu, M, o));
+      double Ssum = pr.y > 0.0 ? pr.y * exp(pr.x - M) : 0.0;
+      for (int o = CL >> 1; o > 0; o >>= 1) Ssum += __shfl_xor_sync(0xffffffffu, Ssum, o);
+      if (act && r == 0) stat[row] = M + log(Ssum);
     }
-    cluster.sync();                                   // nobody leaves while its partials may still be read
+    // no CTA may exit while a peer can still read its partials: arrive now, wait at the end of the kernel
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   } else if (tid < 4 * U) {
     stat[tid] = part[tid].x + log(part[tid].y);
   }
@@ -173,19 +233,24 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
       const double* l = lg + u * 4 * nb;
       const double L1 = l[lb] - stat[u * 4 + 0], L2 = l[nb + lb] - stat[u * 4 + 1];
       const double L3 = l[2 * nb + lb] - stat[u * 4 + 2], L4 = l[3 * nb + lb] - stat[u * 4 + 3];
-      const double Lmax = logaddexp(L1, L3) - ln2;   // ln (S1+S3)/2
-      const double Lmin = logaddexp(L2, L4) - ln2;   // ln (S2+S4)/2
-      v = fmax(Lmax, Lmin);
+      // max( ln (S1+S3)/2, ln (S2+S4)/2 ).  ln(e^a + e^b) lies in [max(a,b), max(a,b) + ln 2], so the pair with the
+      // larger maximum wins outright unless the two maxima are within ln 2 of each other: one evaluation, rarely two.
+      const double h13 = fmax(L1, L3), h24 = fmax(L2, L4);
+      const bool first = h13 >= h24;
+      v = logaddexp(first ? L1 : L2, first ? L3 : L4);
+      if (fabs(h13 - h24) < ln2) v = fmax(v, logaddexp(first ? L2 : L1, first ? L4 : L3));
+      v -= ln2;
       if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + S_prev[unit_of(u) * n2 + bb]);
     }
     S_out[unit_of(u) * n2 + bb] = v;
   }
+  if (CL > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 template <typename T, int D, int U>
 int launch_u(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
              double est_scale, double alpha, int fuse, int mask_first, int CL, int nb, cudaStream_t st) {
-  const size_t smem = sizeof(double) * (4 * size_t(U) * nb);
+  const size_t smem = (sizeof(double) + sizeof(float)) * (4 * size_t(U) * nb);   // fp64 logits + their fp32 copies
   auto kern = score_kernel<T, D, U>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
     return CP_ERR_CUDA;
@@ -217,7 +282,7 @@ int launch_t(const Dims& m, const char* ws, const WsLayout& w, const double* S_p
   const int U = m.g % 4 == 0 ? 4 : (m.g % 2 == 0 ? 2 : 1);
   for (int CL = 1; CL <= 8; CL *= 2) {
     const int nb = (((m.n2 + CL - 1) / CL) + 7) & ~7;
-    if (sizeof(double) * 4 * size_t(U) * nb > budget) continue;
+    if ((sizeof(double) + sizeof(float)) * 4 * size_t(U) * nb > budget) continue;
     if (U == 4) return launch_u<T, D, 4>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
     if (U == 2) return launch_u<T, D, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
     return launch_u<T, D, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
