@@ -455,6 +455,41 @@ def run_sweep(args, cfg):
     print(json.dumps({"sweep": rows, "dense_ms": dense, "config": workload_config(cfg), "data": "synthetic"}))
 
 
+def run_fusion_ablation(args, cfg):
+    """Layer fusion on / off (Algorithm 1, line 14; the "w/o fusion" row of the paper's ablation is alpha = 1)
+    on a stack of seeded layers that share their cluster structure: per layer and per setting, the share of
+    each row's dense softmax mass that the selected blocks hold, and the distance to the dense output."""
+    from paper_2409_12490_b200 import binding as cp
+    from paper_2409_12490_b200.build import build
+    build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    L = args.layers if args.layers else 4
+    variants = [("fusion", cfg), ("no_fusion", cfg.with_(alpha=1.0))]
+    probs = {name: cp.Problem.from_config(c) for name, c in variants}
+    ws = cp.alloc_workspace(probs["fusion"], dev)
+    prev = {name: None for name, _ in variants}
+    rows = []
+    for li in range(L):
+        Q, K, V = (t.to(dev) for t in make_qkv(cfg, layer=li))
+        Od, lsed = cp.dense_attention(probs["fusion"], Q, K, V, ws, want_lse=True)
+        for name, _ in variants:
+            S = cp.estimate(probs[name], Q, K, ws, S_prev=prev[name])
+            idx, cnt = cp.select(probs[name], S, ws)
+            O, lse = cp.attention(probs[name], Q, K, V, idx, cnt, ws, want_lse=True)
+            assert cp.device_status(ws) == 0
+            recall = torch.exp(lse.double() - lsed.double())
+            diff = (O.float() - Od.float()).abs()
+            rows.append({"layer": li, "setting": name, "alpha": probs[name].alpha, "mass_recall_mean": recall.mean().item(),
+                         "mass_recall_median": recall.median().item(),
+                         "mass_recall_p05": recall.flatten().kthvalue(max(1, recall.numel() // 20)).values.item(),
+                         "out_vs_dense_max": diff.max().item(), "out_vs_dense_mean": diff.mean().item()})
+            prev[name] = S
+            del O, lse, idx, cnt, recall, diff
+        del Q, K, V, Od, lsed
+    print(json.dumps({"fusion_ablation": rows, "layers": L, "config": workload_config(cfg), "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -465,6 +500,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="layers in the stack (default: the config's)")
     ap.add_argument("--distinct-layers", type=int, default=2, help="distinct seeded layer inputs cycled through a stack")
     ap.add_argument("--sweep", action="store_true", help="budget x block-size sweep (accuracy vs speed) instead of the bench line")
+    ap.add_argument("--fusion-ablation", action="store_true",
+                    help="layer fusion on/off over a stack of --layers seeded layers (quality diagnostic) instead of the bench line")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -473,6 +510,8 @@ def main():
         run_reference(args, cfg)
     elif args.sweep:
         run_sweep(args, cfg)
+    elif args.fusion_ablation:
+        run_fusion_ablation(args, cfg)
     else:
         run_ours(args, cfg)
 

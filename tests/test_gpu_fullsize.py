@@ -128,3 +128,39 @@ def test_yi_shape_two_layer_chain_at_full_size():
     O_ref, _ = oracle.sparse_attention_rows(Q, K, V, idx.cpu().numpy(), cnt.cpu().numpy(), cfg.segment_size,
                                             cfg.block_size, f32(1.0 / np.sqrt(cfg.head_dim)), rows)
     assert_attention_close(O[rows[:, 0], rows[:, 1], rows[:, 2]], O_ref)
+
+
+def test_paper_operating_point_at_full_size():
+    """The paper's own setting (Section 3.1.3: segment 512, block 32, budget 1024, alpha 0.25) at 128K tokens:
+    n2 = 4096 key blocks, so the score kernel splits them over a thread-block cluster, a gathered K/V tile
+    is four 32-token boxes and the list holds 16 diagonal + 16 past blocks.  Scores with layer fusion
+    (Algorithm 1, line 14) and selection of one KV group against the oracle; attention on sampled rows."""
+    cfg = CONFIGS["paper_128k"]
+    g = cfg.n_q_heads // cfg.n_kv_heads
+    prob = cp.Problem.from_config(cfg)
+    ws = cp.alloc_workspace(prob)
+    kvh = 5
+    hs = slice(kvh * g, (kvh + 1) * g)
+    Q, K, V = make_qkv(cfg)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    S0 = cp.estimate(prob, Qd, Kd, ws)
+    S0_ref = oracle.estimate(Q[:, hs], K[:, kvh:kvh + 1], cfg.segment_size, cfg.block_size, est_scale=f32(cfg.est_scale))
+    compare_scores(S0[:, hs], S0_ref, atol=1e-9)
+    # a second layer on the same inputs, fused onto layer 0's score: the fusion path at this size
+    S1 = cp.estimate(prob, Qd, Kd, ws, S_prev=S0)
+    S1_ref = oracle.estimate(Q[:, hs], K[:, kvh:kvh + 1], cfg.segment_size, cfg.block_size, est_scale=f32(cfg.est_scale),
+                             alpha=f32(cfg.alpha), S_prev=S0_ref)
+    compare_scores(S1[:, hs], S1_ref, atol=1e-9)
+    idx, cnt = cp.select(prob, S1, ws)
+    idx_ref, cnt_ref = oracle.select(S1_ref, cfg.segment_size, cfg.block_size, cfg.budget_blocks)
+    excused, unexcused = compare_selection(idx[:, hs], cnt[:, hs], idx_ref, cnt_ref, S1_ref, cfg.r)
+    assert unexcused == 0
+    O = cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws)
+    assert cp.device_status(ws) == 0
+    rng = np.random.default_rng(4)
+    ts = [0, 31, 32, 511, 512, cfg.seq_len - 1] + [int(t) for t in rng.integers(0, cfg.seq_len, 506)]
+    rows = np.array([(0, kvh * g + int(rng.integers(g)), t) for t in ts], dtype=np.int64)
+    O_ref, _ = oracle.sparse_attention_rows(Q, K, V, idx.cpu().numpy(), cnt.cpu().numpy(), cfg.segment_size,
+                                            cfg.block_size, f32(1.0 / np.sqrt(cfg.head_dim)), rows)
+    mx, mean, _ = assert_attention_close(O[rows[:, 0], rows[:, 1], rows[:, 2]], O_ref)
+    print(f"paper operating point: {excused} excused swaps, attention max abs err {mx:.2e}, mean {mean:.2e}")
