@@ -33,13 +33,32 @@ constexpr int kThreads = 384;   // 3 warpgroups: softmax A, softmax B, {producer
 constexpr int kSmemQ = 0;
 constexpr int kSmemKV = 2 * kTileBytes;
 constexpr int kSmemBar = kSmemKV + kSlots * kTileBytes;
-constexpr int kSmemTotal = kSmemBar + 256 + 1024;   // + barrier block + slack to align the tiles to 1024 bytes
+constexpr int kBarBytes = 512;
+constexpr int kSmemTotal = kSmemBar + kBarBytes + 1024;   // + barrier block + slack to align the tiles to 1024 bytes
 constexpr float kRescaleThreshold = 8.0f;           // in log2 units
 #ifndef CP_EMUL_EVERY
 #define CP_EMUL_EVERY 8
 #endif
 constexpr int kEmulEvery = CP_EMUL_EVERY;           // 0: all exponentials on the MUFU; n: every n-th pair on the FMA pipes
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// One work unit, decoded (the producer warp decodes it once and publishes it to the other warps:
+// the decoding is a chain of integer divisions that would otherwise sit at the start of every unit).
+struct Unit {
+  int b, h, kvh;
+  int q_tok;        // first query row of tile A
+  int n_past;       // listed blocks strictly before the segment
+  int n_past_tiles; // gathered tiles
+  int last_cols;    // valid key columns of the last gathered tile
+  int c_tok, n_cont;// contiguous unmasked tiles: first token, count
+  int d_tok;        // first token of diagonal tile d0 (d1 follows)
+  int T;            // K/V tiles the unit streams
+  int nA, nB;       // tiles query tile A / B consumes (nB = 0: the unit has no tile B)
+  const int32_t* list;
+  int seg_j;
+  int rj;           // diagonal blocks of the segment (r, fewer in a short last segment)
+  int cnt;
+};
 
 struct Bars {
   unsigned long long q_full;
@@ -52,7 +71,7 @@ struct Bars {
   unsigned long long sched_full[2];
   unsigned long long sched_empty[2];
   int sched_unit[2];
-  int sched_cnt[2];
+  Unit sched_u[2];                   // the published unit, decoded; its cnt carries kBadList / kEmptyUnit
   uint32_t tmem_base;
   volatile int abort_flag;
 };
@@ -68,6 +87,7 @@ struct Args {
   float sm_scale;
   int dense;
   int n_units;
+  int o_vec32;                  // O rows are 32-byte aligned: the epilogue may use 32-byte stores
   int withhold_v;               // test hook: the producer never issues V tiles, so a bounded wait must expire
   unsigned int* work_counter;   // next unit to hand out (zeroed by the host before the launch)
 };
@@ -193,6 +213,10 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* w) {   // p must be 32-byte aligned
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+               "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -247,21 +271,6 @@ template <bool kF16> struct Idesc {   // operand format field: 0 = fp16, 1 = bf1
 };
 
 // ---------------------------------------------------------------- unit geometry
-struct Unit {
-  int b, h, kvh;
-  int q_tok;        // first query row of tile A
-  int n_past;       // listed blocks strictly before the segment
-  int n_past_tiles; // gathered tiles
-  int last_cols;    // valid key columns of the last gathered tile
-  int c_tok, n_cont;// contiguous unmasked tiles: first token, count
-  int d_tok;        // first token of diagonal tile d0 (d1 follows)
-  int T;            // K/V tiles the unit streams
-  int nA, nB;       // tiles query tile A / B consumes (nB = 0: the unit has no tile B)
-  const int32_t* list;
-  int seg_j;
-  int rj;           // diagonal blocks of the segment (r, fewer in a short last segment)
-  int cnt;
-};
 
 // Units are ordered KV-head-major so that CTAs resident at the same time share K/V tiles in
 // L2; within a KV head the dense kernel takes the longest rows first.
@@ -356,20 +365,21 @@ __device__ __forceinline__ bool publish_unit(const Args& a, Bars* bars, uint32_t
       cnt = kBadList;
     }
   }
+  u_out->cnt = cnt;
   if (lane == 0) {
     bars->sched_unit[slot] = x;
-    bars->sched_cnt[slot] = cnt;
+    if (x < a.n_units) bars->sched_u[slot] = *u_out;
     mbar_arrive(&bars->sched_full[slot]);
   }
   *x_out = x;
-  u_out->cnt = cnt;
   return true;
 }
-__device__ __forceinline__ bool receive_unit(const Args& a, Bars* bars, uint32_t q, int lane, int* x_out, int* cnt_out) {
+__device__ __forceinline__ bool receive_unit(const Args& a, Bars* bars, uint32_t q, int lane, int* x_out, Unit* u_out) {
   const uint32_t slot = q & 1;
   if (!mbar_wait(&bars->sched_full[slot], (q >> 1) & 1, bars, a.st, 51)) return false;
   *x_out = *reinterpret_cast<volatile int*>(&bars->sched_unit[slot]);
-  *cnt_out = *reinterpret_cast<volatile int*>(&bars->sched_cnt[slot]);
+  if (*x_out < a.n_units) *u_out = bars->sched_u[slot];
+  else u_out->cnt = kEmptyUnit;
   __syncwarp();
   if (lane == 0) mbar_arrive(&bars->sched_empty[slot]);
   return true;
@@ -390,10 +400,10 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
   uint32_t n_units = 0;                               // units finished so far
 
   for (uint32_t q = 0;; ++q) {
-    int x, cnt;
-    if (!receive_unit(a, bars, q, lane, &x, &cnt) || x >= a.n_units || stop_requested(a, bars)) return;
-    if (cnt == kBadList || cnt == kEmptyUnit) continue;
-    const Unit u = decode_unit(a, x, cnt);
+    int x;
+    Unit u;
+    if (!receive_unit(a, bars, q, lane, &x, &u) || x >= a.n_units || bars->abort_flag) return;
+    if (u.cnt == kBadList || u.cnt == kEmptyUnit) continue;
     const int my_tiles = which == 0 ? u.nA : u.nB;
     if (my_tiles == 0) continue;                        // this unit has no tile B
     float m_run = -CUDART_INF, l_run = 0.f;
@@ -498,15 +508,20 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
       uint32_t ov[32];
       tmem_ld32(tO + q * 32, ov);
       tmem_wait_ld();
-      uint4* dst = reinterpret_cast<uint4*>(orow + q * 32);
+      uint32_t w[16];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        uint4 w;
-        w.x = pack2<kF16>(__uint_as_float(ov[8 * i + 0]) * inv, __uint_as_float(ov[8 * i + 1]) * inv);
-        w.y = pack2<kF16>(__uint_as_float(ov[8 * i + 2]) * inv, __uint_as_float(ov[8 * i + 3]) * inv);
-        w.z = pack2<kF16>(__uint_as_float(ov[8 * i + 4]) * inv, __uint_as_float(ov[8 * i + 5]) * inv);
-        w.w = pack2<kF16>(__uint_as_float(ov[8 * i + 6]) * inv, __uint_as_float(ov[8 * i + 7]) * inv);
-        if (t < a.n) dst[i] = w;                     // rows past the end of the sequence (ragged last tile) are dropped
+      for (int i = 0; i < 16; ++i) w[i] = pack2<kF16>(__uint_as_float(ov[2 * i]) * inv, __uint_as_float(ov[2 * i + 1]) * inv);
+      if (t < a.n) {                                 // rows past the end of the sequence (ragged last tile) are dropped
+        if (a.o_vec32) {
+          // 32-byte stores: every store fills whole 32-byte sectors (a thread owns a row, so the lanes of a
+          // store instruction hit 32 different rows; 16-byte stores would touch every sector twice)
+          st_global_v8(orow + q * 32, w);
+          st_global_v8(orow + q * 32 + 16, w + 8);
+        } else {
+          uint4* dst = reinterpret_cast<uint4*>(orow + q * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+        }
       }
     }
     if (a.lse != nullptr && t < a.n)
@@ -527,7 +542,10 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
   Unit u;
   if (!publish_unit(a, bars, 0, lane, &x, &u)) return;
   for (uint32_t q = 0;; ++q) {
-    if (x >= a.n_units || stop_requested(a, bars)) return;
+    if (x >= a.n_units) return;
+    // Only this warp reads the status word in global memory (a round trip the other roles would otherwise
+    // pay at every unit); it tells them through the CTA's abort flag, which their waits poll.
+    if (stop_requested(a, bars)) { bars->abort_flag = 1; return; }
     const Unit u_cur = u;
     if (!publish_unit(a, bars, q + 1, lane, &x, &u)) return;
     if (u_cur.cnt == kBadList || u_cur.cnt == kEmptyUnit) continue;
@@ -603,10 +621,10 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
     return mbar_wait(&bars->kv_full[item % kSlots], (item / kSlots) & 1, bars, a.st, 40);
   };
   for (uint32_t q = 0;; ++q) {
-    int x, cnt;
-    if (!receive_unit(a, bars, q, lane, &x, &cnt) || x >= a.n_units || stop_requested(a, bars)) return;
-    if (cnt == kBadList || cnt == kEmptyUnit) continue;
-    const Unit u = decode_unit(a, x, cnt);
+    int x;
+    Unit u;
+    if (!receive_unit(a, bars, q, lane, &x, &u) || x >= a.n_units || bars->abort_flag) return;
+    if (u.cnt == kBadList || u.cnt == kEmptyUnit) continue;
     const int T = u.T, TA = u.nA;
     const bool hasB = u.nB > 0;
     if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;
@@ -665,6 +683,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t smem_base = (raw + 1023u) & ~1023u;
+  static_assert(sizeof(Bars) <= kBarBytes, "barrier block too small");
   Bars* bars = reinterpret_cast<Bars*>(smem_raw + (smem_base - raw) + kSmemBar);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -768,6 +787,7 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
     return CP_ERR_CUDA;
   a.n_units = int(units);
   a.withhold_v = (p.flags & CP_FLAG_TEST_WITHHOLD_V) ? 1 : 0;
+  a.o_vec32 = (reinterpret_cast<uintptr_t>(O) % 32 == 0 && p.o_stride[0] % 16 == 0 && p.o_stride[1] % 16 == 0 && p.o_stride[2] % 16 == 0) ? 1 : 0;
   a.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(st) + 128);   // inside the status block
   if (cudaMemsetAsync(a.work_counter, 0, sizeof(unsigned int), s) != cudaSuccess) return CP_ERR_CUDA;
   int dev = 0, sms = 0;

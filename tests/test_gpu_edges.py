@@ -224,3 +224,27 @@ def test_repeated_runs_are_bit_identical_and_stay_inside_their_buffers():
         outs.append((S.clone(), idx.clone(), cnt.clone(), O.clone(), lse.clone()))
     for a, b in zip(*outs):
         assert torch.equal(a, b)
+
+
+def test_output_rows_that_are_only_16_byte_aligned():
+    """The tensor-core kernel stores O with 32-byte stores when every row of O starts on a 32-byte boundary and
+    with 16-byte stores otherwise (the interface only asks for 16): an O whose token stride is 136 elements and
+    whose base is offset by 8 elements must receive exactly the bits of the contiguous case, and the padding
+    between its rows must stay untouched."""
+    cfg = BASE.with_(seq_len=768)
+    Q, K, V = make_qkv(cfg)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    O_ref, S, idx, cnt = cp.prefill_layer(prob, Qd, Kd, Vd, ws)
+    canary = 12345.0
+    buf = torch.full((cfg.batch, cfg.n_q_heads, cfg.seq_len, cfg.head_dim + 8), canary, dtype=Qd.dtype, device=Qd.device)
+    O = buf[..., 8:]
+    assert O.data_ptr() % 32 == 16 and O.stride(2) % 16 == 8
+    cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws, O=O)
+    Od = cp.dense_attention(prob, Qd, Kd, Vd, ws)
+    buf2 = torch.full_like(buf, canary)
+    cp.dense_attention(prob, Qd, Kd, Vd, ws, O=buf2[..., 8:])
+    assert cp.device_status(ws) == 0
+    assert torch.equal(O, O_ref) and torch.equal(buf2[..., 8:], Od)
+    assert (buf[..., :8] == canary).all() and (buf2[..., :8] == canary).all()
