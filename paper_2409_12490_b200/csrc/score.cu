@@ -21,13 +21,29 @@ template <> __device__ __forceinline__ double to_f64<float>(float x) { return do
 template <> __device__ __forceinline__ double to_f64<__nv_bfloat16>(__nv_bfloat16 x) { return double(__bfloat162float(x)); }
 template <> __device__ __forceinline__ double to_f64<__half>(__half x) { return double(__half2float(x)); }
 
-// ln(e^a + e^b).  When the smaller term is more than e^-50 below the larger one it cannot change
-// the rounded result (|hi| is at most a few hundred here), so the transcendental pair is skipped.
-__device__ __forceinline__ double logaddexp(double a, double b) {
+// ln(1 + e^-x), x >= 0, from piecewise degree-11 polynomials on intervals of width 1/2 (absolute error 1e-15;
+// the table and how it is made: gen_softplus_table.py).  The library exp + log pair costs several hundred fp64
+// instructions and this function runs once or twice for every element of the score map.
+constexpr int kSpIntervals = 80, kSpCoef = 12, kSpStride = 13;   // stride 13: rows of different intervals hit different banks
+__device__ const double kSoftplusTable[kSpIntervals * kSpCoef] = {
+#include "softplus_table.inc"
+};
+__device__ __forceinline__ double softplus_neg(double x, const double* tab) {
+  if (!(x < 40.0)) return 0.0;              // e^-40 = 4e-18: below the rounding of whatever it is added to
+  const int i = int(x * 2.0);
+  const double t = (x - (0.5 * i + 0.25)) * 4.0;
+  const double* c = tab + i * kSpStride;
+  double p = c[kSpCoef - 1];
+#pragma unroll
+  for (int k = kSpCoef - 2; k >= 0; --k) p = fma(p, t, c[k]);
+  return p;
+}
+// ln(e^a + e^b) = max + ln(1 + e^-(max - min))
+__device__ __forceinline__ double logaddexp(double a, double b, const double* tab) {
   const double hi = fmax(a, b), lo = fmin(a, b);
-  const double d = lo - hi;                 // <= 0, or NaN when both are -inf
-  if (!(d > -50.0)) return hi;
-  return hi + log(1.0 + exp(d));            // absolute error ~2e-16, as good as log1p once it is added to hi
+  const double x = hi - lo;                 // >= 0 (+inf when one term is -inf), or NaN when both are -inf
+  if (!(x >= 0.0)) return hi;
+  return hi + softplus_neg(x, tab);
 }
 
 // Shared memory: logits lg[U][4][nb] (fp64) for the nb key blocks this CTA owns, plus an fp32 copy that
@@ -81,6 +97,9 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   constexpr int SPC = CE / 4;               // MMA k-steps per load
   constexpr int QS = D + 2;                 // row stride of qs in doubles (odd number of 16-byte units: conflict-free)
   __shared__ __align__(16) double qs[8 * QS];   // B operand, row = column index n, laid out [k-step][tig][4 channels]
+  __shared__ double sp_tab[kSpIntervals * kSpStride];
+  for (int e = threadIdx.x; e < kSpIntervals * kSpCoef; e += kThreads)
+    sp_tab[(e / kSpCoef) * kSpStride + e % kSpCoef] = kSoftplusTable[e];
   const int tig = lane & 3, grp = lane >> 2;
   for (int e = tid; e < 8 * D; e += kThreads) {
     const int n = e / D, ch = e % D;        // column n = (head n/2, representative n%2); channel ch
@@ -237,10 +256,10 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
       // larger maximum wins outright unless the two maxima are within ln 2 of each other: one evaluation, rarely two.
       const double h13 = fmax(L1, L3), h24 = fmax(L2, L4);
       const bool first = h13 >= h24;
-      v = logaddexp(first ? L1 : L2, first ? L3 : L4);
-      if (fabs(h13 - h24) < ln2) v = fmax(v, logaddexp(first ? L2 : L1, first ? L4 : L3));
+      v = logaddexp(first ? L1 : L2, first ? L3 : L4, sp_tab);
+      if (fabs(h13 - h24) < ln2) v = fmax(v, logaddexp(first ? L2 : L1, first ? L4 : L3, sp_tab));
       v -= ln2;
-      if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + S_prev[unit_of(u) * n2 + bb]);
+      if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + S_prev[unit_of(u) * n2 + bb], sp_tab);
     }
     S_out[unit_of(u) * n2 + bb] = v;
   }
