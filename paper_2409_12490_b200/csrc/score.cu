@@ -3,8 +3,8 @@
 // key summaries of the group are read and widened to fp64 once and used for all U heads.
 // Per head it forms the four logit rows l1..l4 against every key block, their log-sum-exps, and
 //   ln S = max( ln((S1+S3)/2), ln((S2+S4)/2) ),  mask,  ln(alpha S + (1-alpha) S').
-// The representatives are exact in the input dtype, every product is exact in fp64, so this
-// differs from an fp64 CPU evaluation only by summation order and libm rounding.
+// The representatives are exact in the input dtype and every product is exact in fp64, so this differs
+// from an fp64 CPU evaluation only by summation order, libm rounding and the 1e-15 of the ln(1 + e^-x) table.
 #include <cooperative_groups.h>
 #include <math_constants.h>
 
