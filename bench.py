@@ -32,9 +32,9 @@ METRIC = "128K prefill-attention ms (estimate+select+sparse attention, one layer
 # DRAM bytes (read + write) per launch of the sparse attention kernel, from the ncu captures
 # summarised in profiles/attention_sm100_kernel_C4_counters.md (C4, full size) and
 # profiles/attention_sm100_kernel_C3.md; None for workloads without a capture.
-ATTN_TRAFFIC_BYTES = {"C4": 2.80e9, "C3": 0.635e9}
+ATTN_TRAFFIC_BYTES = {"C4": 2.82e9, "C3": 0.640e9}
 # sm__pipe_tensor_cycles_active (% of peak, elapsed) of the same kernel from the same captures
-ATTN_TENSOR_PIPE_PCT = {"C4": 56.7, "C3": 46.2}
+ATTN_TENSOR_PIPE_PCT = {"C4": 57.7, "C3": 49.1}
 
 
 def load_peaks():
