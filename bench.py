@@ -490,6 +490,42 @@ def run_fusion_ablation(args, cfg):
     print(json.dumps({"fusion_ablation": rows, "layers": L, "config": workload_config(cfg), "data": "synthetic"}))
 
 
+def run_overlap(args, cfg):
+    """Token-wise critical sets (Eq. 3) and how much neighbouring queries share of them (the locality the
+    paper's Section 2 builds on).  With segment = block = 1 Algorithm 1 reduces to softmax(q K^T) per token and
+    Algorithm 2's selection to the per-token top-k, so the library's own estimate + select produce I_i; the
+    overlap |I_i & I_(i+delta)| / k is then counted with torch set operations (a diagnostic, not the hot path).
+    Runs on the first 8192 tokens (the library's limit of key blocks per row) of two query heads."""
+    from paper_2409_12490_b200 import binding as cp
+    from paper_2409_12490_b200.build import build
+    build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n, k = min(cfg.seq_len, 8192), 512
+    Q, K, _ = make_qkv(cfg)
+    g = cfg.n_q_heads // cfg.n_kv_heads
+    Qd = Q[:, :2, :n].contiguous().to(dev)
+    Kd = K[:, :1, :n].contiguous().to(dev) if g >= 2 else K[:, :2, :n].contiguous().to(dev)
+    prob = cp.Problem(cfg.batch, 2, Kd.shape[1], n, cfg.head_dim, 1, 1, k, dtype=Qd.dtype, est_scale=1.0)
+    ws = cp.alloc_workspace(prob, dev)
+    S = cp.estimate(prob, Qd, Kd, ws)
+    idx, cnt = cp.select(prob, S, ws)
+    del S
+    rows = []
+    for h in range(2):
+        member = torch.zeros((n, n), dtype=torch.bool, device=dev)
+        ii = idx[0, h].long()
+        valid = ii >= 0
+        member[torch.arange(n, device=dev)[:, None].expand_as(ii)[valid], ii[valid]] = True
+        for delta in (1, 8, 64, 512, 2048):
+            a, b = member[k:n - delta], member[k + delta:n]          # rows whose lists are full
+            share = (a & b).sum(1).double() / k
+            rows.append({"head": h, "delta": delta, "overlap_mean": share.mean().item(), "overlap_median": share.median().item(),
+                         "overlap_p05": share.kthvalue(max(1, share.numel() // 20)).values.item()})
+        del member
+    print(json.dumps({"token_critical_set_overlap": rows, "k": k, "tokens": n, "config": workload_config(cfg), "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -502,6 +538,8 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="budget x block-size sweep (accuracy vs speed) instead of the bench line")
     ap.add_argument("--fusion-ablation", action="store_true",
                     help="layer fusion on/off over a stack of --layers seeded layers (quality diagnostic) instead of the bench line")
+    ap.add_argument("--overlap", action="store_true",
+                    help="token-wise critical-set overlap between neighbouring queries (Eq. 3; quality diagnostic) instead of the bench line")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -512,6 +550,8 @@ def main():
         run_sweep(args, cfg)
     elif args.fusion_ablation:
         run_fusion_ablation(args, cfg)
+    elif args.overlap:
+        run_overlap(args, cfg)
     else:
         run_ours(args, cfg)
 

@@ -248,3 +248,11 @@ def test_output_rows_that_are_only_16_byte_aligned():
     assert cp.device_status(ws) == 0
     assert torch.equal(O, O_ref) and torch.equal(buf2[..., 8:], Od)
     assert (buf[..., :8] == canary).all() and (buf2[..., :8] == canary).all()
+
+
+def test_single_token_segments_and_blocks_give_token_wise_critical_sets():
+    """segment = block = 1: the four score maps coincide, S is softmax(q K^T) per token and the selection is the
+    token-wise top-k of Eq. 3 (plus the token itself).  Scores, lists and attention over the lists against the oracle."""
+    cfg = BASE.with_(seq_len=640, segment_size=1, block_size=1, budget_tokens=48)
+    Q, K, V = make_qkv(cfg)
+    full_path_vs_oracle(cfg, Q, K, V)
