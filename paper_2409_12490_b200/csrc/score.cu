@@ -111,6 +111,14 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   __syncthreads();
   const int n_tiles = (nloc + 15) / 16;
   for (int t = warp; t < n_tiles; t += kWarps) {
+    if (mask_first && b_lo + t * 16 >= visible) {
+      // normalising over the visible blocks only: a tile of future blocks needs no products at all
+      for (int e = lane; e < 4 * U * 16; e += 32) {
+        const int lb = t * 16 + (e & 15);
+        if (lb < nloc) { lg[(e >> 4) * nb + lb] = -CUDART_INF; lf[(e >> 4) * nb + lb] = -CUDART_INF_F; }
+      }
+      continue;
+    }
     // this lane's two A rows (clamped in a ragged last tile), for the max and the min summaries
     const int blk0 = b_lo + min(t * 16 + grp, nloc - 1), blk1 = b_lo + min(t * 16 + grp + 8, nloc - 1);
     const uint4* src[4] = {reinterpret_cast<const uint4*>(kmx_base + size_t(blk0) * D + tig * KS),
