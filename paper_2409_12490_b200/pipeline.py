@@ -3,8 +3,10 @@ to pinned host memory, pipelined per KV group over three CUDA streams.
 
 Every (batch, KV group) is independent in Algorithm 1 and Algorithm 2, so the layer is cut into
 Hkv sub-problems (g query heads + 1 KV head each).  Group i's host->device copy, the kernels of
-group i-1 and the device->host copy of group i-2's output run concurrently; PCIe is full duplex,
+group i-1 and the device->host copies of earlier outputs run concurrently; PCIe is full duplex,
 so the layer costs about max(bytes in, bytes out) / link rate instead of their sum plus compute.
+Within a group the attention runs head by head and each head's output is copied back as soon as
+it is complete, which shortens the tail after the last input has arrived.
 All arithmetic still runs in the CUDA library (critiprefill_estimate / _select / _attention on
 strided views); this module only moves data and orders streams.
 """
@@ -34,9 +36,11 @@ class HostPipelinedLayer:
         self.S = torch.empty((1, g, self.sub.n1, self.sub.n2), dtype=torch.float64, device=self.dev)
         self.idx = torch.empty((1, g, self.sub.n1, prob.budget_blocks), dtype=torch.int32, device=self.dev)
         self.cnt = torch.empty((1, g, self.sub.n1), dtype=torch.int32, device=self.dev)
+        self.head = cp.Problem(1, 1, 1, prob.seq_len, prob.head_dim, prob.segment_size, prob.block_size,
+                               prob.budget_blocks, prob.dtype, prob.est_scale, prob.sm_scale, prob.alpha, prob.flags)
         self.s_in, self.s_run, self.s_out = (torch.cuda.Stream(self.dev) for _ in range(3))
         self.ev_in = [torch.cuda.Event() for _ in range(prob.n_kv_heads)]
-        self.ev_run = [torch.cuda.Event() for _ in range(prob.n_kv_heads)]
+        self.ev_run = [torch.cuda.Event() for _ in range(prob.n_q_heads)]
 
     def __call__(self, hQ, hK, hV, hO):
         """hQ/hO [1,Hq,n,d], hK/hV [1,Hkv,n,d] pinned host tensors.  Enqueues the whole layer and makes
@@ -57,11 +61,14 @@ class HostPipelinedLayer:
                 Q, K, V, O = self.dQ[:, q], self.dK[:, i:i + 1], self.dV[:, i:i + 1], self.dO[:, q]
                 cp.estimate(self.sub, Q, K, self.ws, S_out=self.S)
                 cp.select(self.sub, self.S, self.ws, idx=self.idx, cnt=self.cnt)
-                cp.attention(self.sub, Q, K, V, self.idx, self.cnt, self.ws, O=O)
-                self.ev_run[i].record(self.s_run)
+                for h in range(g):
+                    one = slice(h, h + 1)
+                    cp.attention(self.head, Q[:, one], K, V, self.idx[:, one], self.cnt[:, one], self.ws, O=O[:, one])
+                    self.ev_run[i * g + h].record(self.s_run)
             with torch.cuda.stream(self.s_out):
-                self.s_out.wait_event(self.ev_run[i])
-                hO[:, q].copy_(self.dO[:, q], non_blocking=True)
+                for h in range(g):
+                    self.s_out.wait_event(self.ev_run[i * g + h])
+                    hO[:, i * g + h:i * g + h + 1].copy_(self.dO[:, i * g + h:i * g + h + 1], non_blocking=True)
         cur.wait_stream(self.s_out)
         cur.wait_stream(self.s_run)
         return hO
