@@ -1,9 +1,9 @@
 // K3: critical block selection (Algorithm 2, line 8).  One CTA per (batch, query head,
 // segment j).  The r diagonal blocks are always taken; the other m = k - r slots go to the
 // strictly-past blocks with the largest score, ties to the larger block index.  Exact:
-// an 8-pass MSB-first radix select on order-preserving 64-bit keys (held in registers) finds
-// the m-th largest score, equal keys are resolved towards larger indices by counting, and an
-// ordered block-wide compaction writes the list ascending.
+// an MSB-first radix select (8 bits per pass, at most 8 passes, usually 3-4) on order-preserving 64-bit
+// keys held in registers finds the m-th largest score, equal keys are resolved towards larger indices by
+// counting, and an ordered block-wide compaction (two scans) writes the list ascending.
 #include "cp_common.cuh"
 
 namespace cp {
@@ -18,7 +18,30 @@ __device__ __forceinline__ unsigned long long ordered_key(double x) {
   return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// KPT = keys per thread; block b of the row lives in thread b % 256, slot b / 256.
+// Block-wide exclusive scan of one int per thread (256 threads); *total receives the sum.  Two barriers.
+__device__ __forceinline__ int block_exclusive_scan(int v, int lane, int warp, int* warp_tot, int* total) {
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  int before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    const int t = warp_tot[w];
+    before += w < warp ? t : 0;
+    all += t;
+  }
+  __syncthreads();                      // warp_tot may be reused by the next scan
+  *total = all;
+  return before + incl - v;
+}
+
+// KPT = keys per thread; thread t owns the KPT consecutive blocks [t*KPT, (t+1)*KPT), so the ordered
+// compaction at the end is two block-wide scans instead of a barrier-separated step per key slot.
 template <int KPT>
 __global__ void __launch_bounds__(kThreads)
 select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* __restrict__ cnt,
@@ -26,9 +49,8 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
   __shared__ unsigned int hist[256];
   __shared__ int warp_sum[kWarps];
   __shared__ unsigned long long prefix_sh;
-  __shared__ int remaining_sh;
-  __shared__ int warp_tot[2][kWarps];
-  __shared__ int base_sh[2];
+  __shared__ int remaining_sh, bin_count_sh;
+  __shared__ int warp_tot[kWarps];
 
   const int unit = blockIdx.x;
   const int j = unit % n1;
@@ -54,30 +76,31 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
     return;
   }
 
+  const int b0 = tid * KPT;                  // first block owned by this thread
   unsigned long long key[KPT];
 #pragma unroll
-  for (int s = 0; s < KPT; ++s) {
-    const int b = s * kThreads + tid;
-    key[s] = b < past ? ordered_key(row[b]) : 0ull;
-  }
+  for (int s = 0; s < KPT; ++s) key[s] = b0 + s < past ? ordered_key(__ldg(row + b0 + s)) : 0ull;
+  hist[tid] = 0;
+  __syncthreads();
 
   // ---- radix select: key of the m-th largest past score --------------------------------
+  // MSB-first, 8 bits per pass.  A pass ends the search early when the bin that holds the m-th largest key
+  // holds exactly as many keys as are still to be taken: then every key of that bin (and above) is selected
+  // and no tie has to be resolved.  With distinct scores this happens after 3-4 of the 8 passes.
   unsigned long long prefix = 0;   // bits decided so far (high bits)
   int remaining = m;               // how many still to take among keys matching the prefix
+  bool all_of_bin = false;
   for (int pass = 0; pass < 8; ++pass) {
     const int shift = 56 - 8 * pass;
-    hist[tid] = 0;
-    __syncthreads();
     const unsigned long long himask = pass == 0 ? 0ull : (~0ull << (shift + 8));
 #pragma unroll
-    for (int s = 0; s < KPT; ++s) {
-      const int b = s * kThreads + tid;
-      if (b < past && (key[s] & himask) == prefix) atomicAdd(&hist[(key[s] >> shift) & 0xff], 1u);
-    }
+    for (int s = 0; s < KPT; ++s)
+      if (b0 + s < past && (key[s] & himask) == prefix) atomicAdd(&hist[(key[s] >> shift) & 0xff], 1u);
     __syncthreads();
     // suffix sums over the 256 bins: thread t owns bin t; above(t) = keys with a larger digit
     const int mine = int(hist[tid]);
-    int incl = mine;   // inclusive suffix sum within the warp (towards higher lanes)
+    hist[tid] = 0;                 // only its owner reads a bin, so it can be cleared for the next pass right away
+    int incl = mine;               // inclusive suffix sum within the warp (towards higher lanes)
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int v = __shfl_down_sync(0xffffffffu, incl, o);
@@ -90,56 +113,47 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
     if (above < remaining && remaining <= above + mine) {   // exactly one bin satisfies this
       prefix_sh = prefix | ((unsigned long long)tid << shift);
       remaining_sh = remaining - above;
+      bin_count_sh = mine;
     }
     __syncthreads();
     prefix = prefix_sh;
     remaining = remaining_sh;
+    if (bin_count_sh == remaining) { all_of_bin = true; break; }   // uniform: read from shared memory by all
   }
-  const unsigned long long thr = prefix;   // the m-th largest key
-  const int need_eq = remaining;           // of the keys equal to thr, take this many (largest indices)
-
-  // total number of keys equal to the threshold
-  if (tid == 0) base_sh[0] = 0;
-  __syncthreads();
-  int eq_local = 0;
-#pragma unroll
-  for (int s = 0; s < KPT; ++s) eq_local += (s * kThreads + tid < past) && key[s] == thr;
-  for (int o = 16; o > 0; o >>= 1) eq_local += __shfl_xor_sync(0xffffffffu, eq_local, o);
-  if (lane == 0 && eq_local) atomicAdd(&base_sh[0], eq_local);
-  __syncthreads();
-  const int eq_skip = base_sh[0] - need_eq;   // equal keys with the smallest indices are dropped
-  __syncthreads();
-
-  // ---- ordered compaction -----------------------------------------------------------------
-  if (tid == 0) { base_sh[0] = 0; base_sh[1] = 0; }   // [0]: written so far, [1]: equals seen so far
-  __syncthreads();
+  // all_of_bin: take every key >= prefix (its undecided low bits are zero).  Otherwise prefix is the m-th
+  // largest key itself: take the keys above it and, of the keys equal to it, the `remaining` largest indices.
+  const unsigned long long thr = prefix;
+  int n_gt = 0, n_eq = 0;
 #pragma unroll
   for (int s = 0; s < KPT; ++s) {
-    const int b0 = s * kThreads;
-    if (b0 >= past) break;
-    const int b = b0 + tid;
-    const bool in = b < past;
-    const bool gt = in && key[s] > thr, eq = in && key[s] == thr;
-    const unsigned eq_ballot = __ballot_sync(0xffffffffu, eq);
-    const int eq_before_warp = __popc(eq_ballot & ((1u << lane) - 1));
-    if (lane == 0) warp_tot[1][warp] = __popc(eq_ballot);
-    __syncthreads();
-    int eq_before = base_sh[1] + eq_before_warp;
-    for (int w = 0; w < warp; ++w) eq_before += warp_tot[1][w];
-    const bool take = gt || (eq && eq_before >= eq_skip);
-    const unsigned tk_ballot = __ballot_sync(0xffffffffu, take);
-    if (lane == 0) warp_tot[0][warp] = __popc(tk_ballot);
-    __syncthreads();
-    int pos = base_sh[0] + __popc(tk_ballot & ((1u << lane) - 1));
-    for (int w = 0; w < warp; ++w) pos += warp_tot[0][w];
-    if (take && pos < m) out[pos] = b;
-    __syncthreads();
-    if (tid == 0) {
-      int a = 0, e = 0;
-      for (int w = 0; w < kWarps; ++w) { a += warp_tot[0][w]; e += warp_tot[1][w]; }
-      base_sh[0] += a; base_sh[1] += e;
-    }
-    __syncthreads();
+    const bool in = b0 + s < past;
+    n_gt += in && (all_of_bin ? key[s] >= thr : key[s] > thr);
+    n_eq += in && !all_of_bin && key[s] == thr;
+  }
+  int eq_before = 0, eq_skip = 0;
+  if (!all_of_bin) {                         // uniform branch
+    int total_eq;
+    eq_before = block_exclusive_scan(n_eq, lane, warp, warp_tot, &total_eq);
+    eq_skip = total_eq - remaining;          // equal keys with the smallest indices are dropped
+  }
+  int n_take = n_gt;
+  if (!all_of_bin) {
+#pragma unroll
+    for (int s = 0, e = eq_before; s < KPT; ++s)
+      if (b0 + s < past && key[s] == thr) { n_take += e >= eq_skip; ++e; }
+  }
+
+  // ---- ordered compaction: blocks are owned in index order, so positions are an exclusive scan ----
+  int total_take;
+  int pos = block_exclusive_scan(n_take, lane, warp, warp_tot, &total_take);
+#pragma unroll
+  for (int s = 0, e = eq_before; s < KPT; ++s) {
+    if (b0 + s >= past) break;
+    bool take;
+    if (all_of_bin) take = key[s] >= thr;
+    else if (key[s] == thr) { take = e >= eq_skip; ++e; }
+    else take = key[s] > thr;
+    if (take) { if (pos < m) out[pos] = b0 + s; ++pos; }
   }
   for (int i = tid; i < rj; i += kThreads) out[m + i] = past + i;   // diagonal blocks
   if (tid == 0) cnt[unit] = k;
