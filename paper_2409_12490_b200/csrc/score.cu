@@ -101,6 +101,12 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   for (int e = threadIdx.x; e < kSpIntervals * kSpCoef; e += kThreads)
     sp_tab[(e / kSpCoef) * kSpStride + e % kSpCoef] = kSoftplusTable[e];
   const int tig = lane & 3, grp = lane >> 2;
+  if (fuse && (lane & 15) == 0) {
+    // the previous layer's scores of this CTA's elements are read once, at the very end: start them towards L2 now
+    for (int u = 0; u < U; ++u)
+      for (int lb = tid; lb < nloc && b_lo + lb < visible; lb += kThreads)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(S_prev + unit_of(u) * n2 + b_lo + lb));
+  }
   for (int e = tid; e < 8 * D; e += kThreads) {
     const int n = e / D, ch = e % D;        // column n = (head n/2, representative n%2); channel ch
     const int u = n >> 1, rep = n & 1;
@@ -248,28 +254,31 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   }
   __syncthreads();
 
-  // combine (lines 11-12), mask (13), fusion (14) over this CTA's blocks of the U rows, flattened
+  // combine (lines 11-12), mask (13), fusion (14) over this CTA's blocks of the U rows
   const double ln2 = 0.693147180559945309417232121458;
+#pragma unroll 1
+  for (int u = 0; u < U; ++u) {
+    const double* l = lg + u * 4 * nb;
+    const double st1 = stat[u * 4 + 0], st2 = stat[u * 4 + 1], st3 = stat[u * 4 + 2], st4 = stat[u * 4 + 3];
+    const size_t out_row = unit_of(u) * n2 + b_lo;
 #pragma unroll 2
-  for (int e = tid; e < U * nloc; e += kThreads) {
-    const int u = e / nloc, lb = e - u * nloc, bb = b_lo + lb;
-    double v;
-    if (bb >= visible) {
-      v = -CUDART_INF;
-    } else {
-      const double* l = lg + u * 4 * nb;
-      const double L1 = l[lb] - stat[u * 4 + 0], L2 = l[nb + lb] - stat[u * 4 + 1];
-      const double L3 = l[2 * nb + lb] - stat[u * 4 + 2], L4 = l[3 * nb + lb] - stat[u * 4 + 3];
-      // max( ln (S1+S3)/2, ln (S2+S4)/2 ).  ln(e^a + e^b) lies in [max(a,b), max(a,b) + ln 2], so the pair with the
-      // larger maximum wins outright unless the two maxima are within ln 2 of each other: one evaluation, rarely two.
-      const double h13 = fmax(L1, L3), h24 = fmax(L2, L4);
-      const bool first = h13 >= h24;
-      v = logaddexp(first ? L1 : L2, first ? L3 : L4, sp_tab);
-      if (fabs(h13 - h24) < ln2) v = fmax(v, logaddexp(first ? L2 : L1, first ? L4 : L3, sp_tab));
-      v -= ln2;
-      if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + S_prev[unit_of(u) * n2 + bb], sp_tab);
+    for (int lb = tid; lb < nloc; lb += kThreads) {
+      double v;
+      if (b_lo + lb >= visible) {
+        v = -CUDART_INF;
+      } else {
+        const double L1 = l[lb] - st1, L2 = l[nb + lb] - st2, L3 = l[2 * nb + lb] - st3, L4 = l[3 * nb + lb] - st4;
+        // max( ln (S1+S3)/2, ln (S2+S4)/2 ).  ln(e^a + e^b) lies in [max(a,b), max(a,b) + ln 2], so the pair with the
+        // larger maximum wins outright unless the two maxima are within ln 2 of each other: one evaluation, rarely two.
+        const double h13 = fmax(L1, L3), h24 = fmax(L2, L4);
+        const bool first = h13 >= h24;
+        v = logaddexp(first ? L1 : L2, first ? L3 : L4, sp_tab);
+        if (fabs(h13 - h24) < ln2) v = fmax(v, logaddexp(first ? L2 : L1, first ? L4 : L3, sp_tab));
+        v -= ln2;
+        if (fuse) v = logaddexp(ln_alpha + v, ln_1m_alpha + S_prev[out_row + lb], sp_tab);
+      }
+      S_out[out_row + lb] = v;
     }
-    S_out[unit_of(u) * n2 + bb] = v;
   }
   if (CL > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
