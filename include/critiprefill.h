@@ -13,6 +13,9 @@
  *   - Calls validate their arguments on the host, enqueue kernels on `cuda_stream`
  *     (a cudaStream_t passed as void*; NULL = the default stream) and return without
  *     synchronising.  Outputs are valid once the stream reaches that point.
+ *     The calls (critiprefill_device_status excepted) only enqueue kernels and one small memset, so a stream
+ *     that is being captured into a CUDA graph may carry them; the graph then refers to the buffers given at
+ *     capture time (tensor maps are encoded on the host from those pointers).
  *   - Return value: a cp_status.  Conditions only the device can see (a block list that
  *     breaks its contract, a pipeline wait that ran out) are recorded in the first word of
  *     the workspace; read it with critiprefill_device_status.  Kernels never trap or assert.

@@ -256,3 +256,35 @@ def test_single_token_segments_and_blocks_give_token_wise_critical_sets():
     cfg = BASE.with_(seq_len=640, segment_size=1, block_size=1, budget_tokens=48)
     Q, K, V = make_qkv(cfg)
     full_path_vs_oracle(cfg, Q, K, V)
+
+
+def test_layer_replays_from_a_cuda_graph():
+    """estimate + select + attention captured once into a CUDA graph (the library only enqueues kernels and one
+    memset on the caller's stream, and encodes its tensor maps on the host) and replayed on new inputs written
+    into the same buffers: every replay must equal the eager result for those inputs."""
+    cfg = BASE.with_(seq_len=1536)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    Q0, K0, V0 = to_dev(*make_qkv(cfg))
+    Q, K, V = Q0.clone(), K0.clone(), V0.clone()
+    O_eager, S_eager, idx_eager, cnt_eager = cp.prefill_layer(prob, Q, K, V, ws)
+    S, idx, cnt, O = torch.empty_like(S_eager), torch.empty_like(idx_eager), torch.empty_like(cnt_eager), torch.empty_like(O_eager)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            cp.estimate(prob, Q, K, ws, S_out=S)
+            cp.select(prob, S, ws, idx=idx, cnt=cnt)
+            cp.attention(prob, Q, K, V, idx, cnt, ws, O=O)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(O, O_eager) and torch.equal(idx, idx_eager) and torch.equal(S, S_eager)
+    Q1, K1, V1 = to_dev(*make_qkv(cfg, layer=1))
+    O1_eager, _, idx1_eager, _ = cp.prefill_layer(prob, Q1, K1, V1, ws)
+    Q.copy_(Q1); K.copy_(K1); V.copy_(V1)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert cp.device_status(ws) == 0
+    assert torch.equal(O, O1_eager) and torch.equal(idx, idx1_eager)
+    assert not torch.equal(O1_eager, O_eager)
