@@ -133,9 +133,10 @@ def physical_gpu_index(local: int) -> int:
 
 
 # ----------------------------------------------------------------------------- reference arm
-def oracle_step(cfg, Q, K, V, head, n_rows, seed):
+def oracle_step(cfg, Q, K, V, head, n_rows, seed, keep=None):
     """A bounded sample of one layer pass on the CPU oracle: Algorithm 1 + selection for one
-    query head, Algorithm 2 for `n_rows` random rows of it.  Returns (seconds_est_sel, seconds_attn)."""
+    query head, Algorithm 2 for `n_rows` random rows of it.  Returns (seconds_est_sel, seconds_attn);
+    with a dict in `keep` the oracle's results are left there for a comparison with the CUDA path."""
     import oracle
     g = cfg.n_q_heads // cfg.n_kv_heads
     q, k, v = Q[:, head:head + 1], K[:, head // g:head // g + 1], V[:, head // g:head // g + 1]
@@ -146,10 +147,29 @@ def oracle_step(cfg, Q, K, V, head, n_rows, seed):
     rng = np.random.default_rng(seed)
     rows = np.stack([np.zeros(n_rows, np.int64), np.zeros(n_rows, np.int64),
                      rng.integers(0, cfg.seq_len, n_rows)], axis=1)
-    oracle.sparse_attention_rows(q, k, v, idx, cnt, cfg.segment_size, cfg.block_size,
-                                 1.0 / math.sqrt(cfg.head_dim), rows)
+    O_rows, _ = oracle.sparse_attention_rows(q, k, v, idx, cnt, cfg.segment_size, cfg.block_size,
+                                             1.0 / math.sqrt(cfg.head_dim), rows)
     t2 = time.perf_counter()
+    if keep is not None:
+        keep.update(S=S, idx=idx, cnt=cnt, rows=rows, O_rows=O_rows)
     return t1 - t0, t2 - t1
+
+
+def parity_summary(head, ref, S, idx, cnt, O):
+    """The timed outputs of the CUDA path against what the oracle sample computed for the same head."""
+    S_gpu = S[:, head:head + 1].cpu().numpy()
+    fin = np.isfinite(ref["S"])
+    same_mask = bool(np.array_equal(np.isfinite(S_gpu), fin))
+    idx_gpu, cnt_gpu = idx[:, head:head + 1].cpu().numpy(), cnt[:, head:head + 1].cpu().numpy()
+    units = int(np.prod(cnt_gpu.shape))
+    equal = np.all(idx_gpu == ref["idx"], axis=-1) & (cnt_gpu == ref["cnt"])
+    rows = ref["rows"]
+    O_gpu = O[rows[:, 0], head, rows[:, 2]].float().cpu().numpy().astype(np.float64)
+    err = np.abs(O_gpu - ref["O_rows"])
+    return {"head": head, "ln_S_max_abs_diff": float(np.abs(S_gpu[fin] - ref["S"][fin]).max()) if same_mask else None,
+            "mask_equal": same_mask, "selection_units": units, "selection_units_differing": int(units - equal.sum()),
+            "attention_rows": int(len(rows)), "attention_max_abs_err": float(err.max()), "attention_mean_abs_err": float(err.mean()),
+            "note": "oracle = fp64 CPU restatement of Algorithms 1-2; attention rows use the oracle's lists"}
 
 
 def oracle_ms_per_layer(cfg, t_est, t_attn, n_rows):
@@ -397,7 +417,10 @@ def run_ours(args, cfg):
         import oracle.build
         oracle.build.build()
         n_rows = min(4 * cfg.seq_len, 262144)      # about 10 s of oracle work on 16 cores at C4
-        te, ta = oracle_step(cfg, Q, K, V, 5 % cfg.n_q_heads, n_rows, 0)
+        ref = {} if L == 1 else None
+        te, ta = oracle_step(cfg, Q, K, V, 5 % cfg.n_q_heads, n_rows, 0, keep=ref)
+        if ref is not None:
+            out["parity"] = parity_summary(5 % cfg.n_q_heads, ref, S, idx, cnt, O)
         out["cpu_baseline"] = {
             "value": oracle_ms_per_layer(cfg, te, ta, n_rows), "unit": "ms", "cores": os.cpu_count(), "kind": "oracle",
             "sample": f"Algorithm 1 + selection for 1 of {cfg.n_q_heads} query heads ({te:.1f} s, numpy) and Algorithm 2 "
