@@ -112,7 +112,9 @@ def estimate(Q, K, segment_size: int, block_size: int, *, est_scale: float = 1.0
     Lmin = _logaddexp(L[1], L[3]) - LN2                                          #          (S2+S4)/2
     Lg = np.maximum(Lmax, Lmin)                                                  # line 12
     Lg = np.where(masked, -np.inf, Lg)                                           # line 13
-    if S_prev is not None and alpha != 1.0:                                      # line 14
+    if S_prev is not None:                                                       # line 14
         Lprev = np.asarray(S_prev, dtype=np.float64)
-        Lg = _logaddexp(np.log(alpha) + Lg, np.log1p(-alpha) + Lprev)            # ln(a*S + (1-a)*S')
+        with np.errstate(divide="ignore"):                                       # alpha = 0 or 1: one weight is ln 0 = -inf
+            ln_a, ln_1ma = np.log(np.float64(alpha)), np.log1p(-np.float64(alpha))
+        Lg = _logaddexp(ln_a + Lg, ln_1ma + Lprev)                               # ln(a*S + (1-a)*S')
     return Lg
