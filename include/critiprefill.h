@@ -9,7 +9,8 @@
  * General conventions
  *   - Every pointer argument except `p`, `bytes_out` and `status_out` is a DEVICE pointer
  *     owned by the caller.  The library allocates no device memory, frees nothing and keeps
- *     no state between calls.
+ *     no state between calls (one exception: critiprefill_estimate_static remembers, per device,
+ *     the address of its built-in scratch array; see there).
  *   - Calls validate their arguments on the host, enqueue kernels on `cuda_stream`
  *     (a cudaStream_t passed as void*; NULL = the default stream) and return without
  *     synchronising.  Outputs are valid once the stream reaches that point.
@@ -74,7 +75,7 @@ typedef struct {
   float est_scale; /* multiplies the four estimation logits; 1.0 = Algorithm 1 as printed */
   float sm_scale;  /* attention logit scale, 1/sqrt(head_dim) in Eq. 2 / Algorithm 2 line 10 */
   float alpha;     /* layer-fusion weight of the current layer (Algorithm 1 line 14; 0.25 in
-                      Section 3.1.3); ignored when S_prev is NULL */
+                      Section 3.1.3), in [0, 1] (else CP_ERR_SHAPE); ignored when S_prev is NULL */
   int32_t reserved;
 } cp_params;
 
@@ -107,7 +108,10 @@ int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, cons
  * synchronisation, a plug-in bound by its host's allocation rules.  Same arguments, results
  * and arithmetic as critiprefill_estimate, minus `ws`: the summaries go to an 8 MiB array
  * that is part of the library's device image (critiprefill_static_scratch_bytes(); every GPU
- * that loads the library holds it until the process exits).
+ * that loads the library holds it until the process exits).  8 MiB holds, for instance, 128K
+ * tokens of 32 query / 8 KV heads at segment 1024 / block 128, but not at segment 512 / block 32.
+ *   - The resolved address is cached per device for the life of the process; do not call this
+ *     entry point again on a device after a cudaDeviceReset of that device.
  *   - Problems whose critiprefill_workspace_bytes exceeds that size return
  *     CP_ERR_STATIC_LIMIT and launch nothing.
  *   - The call allocates and frees nothing (no cudaMalloc/cudaFree, no allocating library

@@ -69,6 +69,7 @@ int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, cons
   if (rc != CP_OK) return rc;
   if (!Q || !K || !S_out) return CP_ERR_NULL;
   if (!aligned16(Q) || !aligned16(K) || S_out == S_prev) return CP_ERR_SHAPE;
+  if (S_prev != nullptr && !(p->alpha >= 0.0f && p->alpha <= 1.0f)) return CP_ERR_SHAPE;   // line 14 is a convex combination (NaN fails too)
   if (m.n2 > kMaxBlocksN2) return CP_ERR_UNSUPPORTED;
   if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

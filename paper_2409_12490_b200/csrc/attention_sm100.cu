@@ -41,6 +41,7 @@ constexpr float kRescaleThreshold = 8.0f;           // in log2 units
 #endif
 constexpr int kEmulEvery = CP_EMUL_EVERY;           // 0: all exponentials on the MUFU; n: every n-th pair on the FMA pipes
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr int kRegPoolNeeded = 256 * 216 + 128 * 64;   // registers the roles hold after setmaxnreg (softmax 216, producer/MMA 64)
 
 // One work unit, decoded (the producer warp decodes it once and publishes it to the other warps:
 // the decoding is a chain of integer divisions that would otherwise sit at the start of every unit).
@@ -715,7 +716,7 @@ attention_sm100_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
 
   // Register re-partition.  The pool is what the CTA was launched with (384 threads x 168):
   // 256 x 216 + 128 x 64 = 63488 fits; asking for more than the pool would block forever.
-  static_assert(256 * 216 + 128 * 64 <= kThreads * 168, "setmaxnreg budget exceeds the launch allocation");
+  static_assert(kRegPoolNeeded <= kThreads * 168, "setmaxnreg budget exceeds the launch allocation");
   if (warp < 8) {
     reg_inc<216>();
     softmax_role<kF16>(a, bars, warp >> 2, warp & 3, lane);
@@ -791,6 +792,16 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
                                 : (long long)m.B * m.Hq * m.n1 * ((m.seg / kTile + 1) / 2);
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
   auto kern = f16 ? attention_sm100_kernel<true> : attention_sm100_kernel<false>;
+  // setmaxnreg.inc blocks forever when the CTA's register pool (threads x registers the kernel was compiled
+  // to) is smaller than what the roles ask for, and no bounded wait covers that: check the real allocation of
+  // this build once per variant and refuse to launch instead.
+  static int regs_ok[2] = {0, 0};   // 0 = not checked yet, 1 = fits, -1 = does not fit
+  if (regs_ok[f16] == 0) {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return CP_ERR_CUDA;
+    regs_ok[f16] = (fa.numRegs * kThreads >= kRegPoolNeeded) ? 1 : -1;
+  }
+  if (regs_ok[f16] < 0) return CP_ERR_UNSUPPORTED;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal) != cudaSuccess)
     return CP_ERR_CUDA;
   a.n_units = int(units);

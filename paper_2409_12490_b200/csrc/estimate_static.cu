@@ -14,7 +14,10 @@
 
 namespace {
 
-constexpr size_t kStaticScratchBytes = size_t(8) << 20;   // 8 MiB: covers the 128K-token configurations
+// 8 MiB.  Enough for 128K tokens of 32 query / 8 KV heads at segment 1024 / block 128 (6 MiB of summaries) and for the
+// 32 / 4-head shape (4 MiB); NOT enough for segment 512 / block 32 at 128K tokens (4 MiB of query + 16 MiB of key
+// summaries), which gets CP_ERR_STATIC_LIMIT.
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;
 constexpr int kMaxDevices = 64;
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress;
@@ -24,7 +27,9 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 std::mutex g_mutex;
 void* g_scratch_ptr[kMaxDevices] = {nullptr};
 
-// Device address of the array on the current device, resolved once per device.
+// Device address of the array on the current device, resolved once per device and cached for the life of
+// the process.  cudaDeviceReset unloads the library's device image, after which a cached address is stale:
+// this entry point must not be used across a reset of a device it has already served.
 int static_scratch(void** out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CP_ERR_CUDA;
@@ -50,6 +55,7 @@ extern "C" int critiprefill_estimate_static(const cp_params* p, const void* Q, c
   if (!Q || !K || !S_out) return CP_ERR_NULL;
   if ((reinterpret_cast<uintptr_t>(Q) & 15u) || (reinterpret_cast<uintptr_t>(K) & 15u) || S_out == S_prev)
     return CP_ERR_SHAPE;
+  if (S_prev != nullptr && !(p->alpha >= 0.0f && p->alpha <= 1.0f)) return CP_ERR_SHAPE;
   const Dims m = make_dims(*p);
   if (m.n2 > kMaxBlocksN2) return CP_ERR_UNSUPPORTED;
   void* scratch = nullptr;
