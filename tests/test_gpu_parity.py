@@ -55,6 +55,23 @@ def test_estimate_variants(est_scale, flags):
     compare_scores(S, oracle_scores(cfg, Q, K, mask_before_softmax=bool(flags)))
 
 
+def test_alpha_one_with_previous_scores_is_the_unfused_score():
+    """alpha = 1 with a non-NULL S_prev (the paper's "w/o fusion" setting run through the fusing call): the kernel
+    must return the unfused ln S.  The oracle evaluates line 14 in full, logaddexp(ln 1 + ln S, ln 0 + ln S')."""
+    cfg = SMALL_BF16.with_(alpha=1.0)
+    Q, K, _ = make_qkv(cfg)
+    rng = np.random.default_rng(3)
+    S_prev = oracle_scores(cfg, *make_qkv(cfg, layer=1)[:2]) + rng.standard_normal((1, 4, cfg.n1, cfg.n2))
+    _, _, S, idx, cnt = run_estimate_select(cfg, Q, K, S_prev=S_prev)
+    S_ref = oracle_scores(cfg, Q, K, S_prev=S_prev)
+    assert np.array_equal(S_ref, oracle_scores(cfg, Q, K))          # identity on the oracle side, through the formula
+    compare_scores(S, S_ref)
+    # alpha = 0 is the other end: the previous layer's score is returned
+    cfg0 = SMALL_BF16.with_(alpha=0.0)
+    _, _, S0, _, _ = run_estimate_select(cfg0, Q, K, S_prev=S_prev)
+    compare_scores(S0, oracle_scores(cfg0, Q, K, S_prev=S_prev))
+
+
 def test_attention_fp32_simt_matches_oracle():
     cfg = CONFIGS["C1"]
     Q, K, V = make_qkv(cfg)
@@ -184,3 +201,8 @@ def test_host_side_argument_errors():
     with pytest.raises(cp.CritiPrefillError) as e:
         cp.workspace_bytes(bad)
     assert e.value.status == 2
+    S_prev = torch.zeros((1, 4, cfg.n1, cfg.n2), dtype=torch.float64, device="cuda")
+    for alpha in (-0.1, 1.5, float("nan")):                        # line 14 is a convex combination
+        with pytest.raises(cp.CritiPrefillError) as e:
+            cp.estimate(cp.Problem.from_config(cfg.with_(alpha=alpha)), Q, K, ws, S_prev=S_prev)
+        assert e.value.status == 2
