@@ -74,7 +74,7 @@ int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, cons
   if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if ((rc = launch_summarize(*p, m, Q, K, static_cast<char*>(ws), s)) != CP_OK) return rc;
-  return launch_score(*p, m, static_cast<const char*>(ws), S_prev, S_out, s);
+  return launch_score(*p, m, static_cast<char*>(ws), S_prev, S_out, s);
 }
 
 int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws, size_t ws_bytes,

@@ -28,9 +28,11 @@ inline Dims make_dims(const cp_params& p) {
   return m;
 }
 
-// Workspace layout: [status 256 B][Qmax][Qmin][Kmax][Kmin], summaries in the input dtype.
+// Workspace layout: [status 256 B][Qmax][Qmin][Kmax][Kmin][stats][kabs]: summaries in the input dtype;
+// stats = the four log-sum-exps of every (head, segment) row, [B,Hq,n1,4] fp64; kabs = largest magnitude
+// in each key block's summaries, [B,Hkv,n2] fp32.
 struct WsLayout {
-  size_t qmax, qmin, kmax, kmin, total;
+  size_t qmax, qmin, kmax, kmin, stats, kabs, total;
 };
 inline WsLayout ws_layout(const Dims& m) {
   auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
@@ -38,7 +40,9 @@ inline WsLayout ws_layout(const Dims& m) {
   size_t qs = up(size_t(m.B) * m.Hq * m.n1 * m.d * m.es);
   size_t ks = up(size_t(m.B) * m.Hkv * m.n2 * m.d * m.es);
   w.qmax = kStatusBytes; w.qmin = w.qmax + qs; w.kmax = w.qmin + qs; w.kmin = w.kmax + ks;
-  w.total = w.kmin + ks;
+  w.stats = w.kmin + ks;
+  w.kabs = w.stats + up(size_t(m.B) * m.Hq * m.n1 * 4 * sizeof(double));
+  w.total = w.kabs + up(size_t(m.B) * m.Hkv * m.n2 * sizeof(float));
   return w;
 }
 
@@ -60,8 +64,11 @@ __device__ __forceinline__ void report(DeviceStatus* st, int code, int where, in
 // Kernel launchers (each returns a cp_status).
 int launch_summarize(const cp_params& p, const Dims& m, const void* Q, const void* K, char* ws,
                      cudaStream_t s);
-int launch_score(const cp_params& p, const Dims& m, const char* ws, const double* S_prev,
+int launch_score(const cp_params& p, const Dims& m, char* ws, const double* S_prev,
                  double* S_out, cudaStream_t s);
+int launch_lse(const cp_params& p, const Dims& m, char* ws, cudaStream_t s);   // stats region of ws <- row log-sum-exps
+int launch_score_generic(const cp_params& p, const Dims& m, const char* ws, const double* S_prev,
+                         double* S_out, double* stats_out, cudaStream_t s);
 int launch_select(const cp_params& p, const Dims& m, const double* S, int32_t* idx, int32_t* cnt,
                   cudaStream_t s);
 int launch_attention_simt(const cp_params& p, const Dims& m, const void* Q, const void* K,

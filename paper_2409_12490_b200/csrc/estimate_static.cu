@@ -65,7 +65,7 @@ extern "C" int critiprefill_estimate_static(const cp_params* p, const void* Q, c
   // before they are read; the 256-byte status head is the only part that must start at zero.
   if (cudaMemsetAsync(scratch, 0, kStatusBytes, s) != cudaSuccess) return CP_ERR_CUDA;
   if ((rc = launch_summarize(*p, m, Q, K, static_cast<char*>(scratch), s)) != CP_OK) return rc;
-  return launch_score(*p, m, static_cast<const char*>(scratch), S_prev, S_out, s);
+  return launch_score(*p, m, static_cast<char*>(scratch), S_prev, S_out, s);
 }
 
 extern "C" size_t critiprefill_static_scratch_bytes(void) { return kStaticScratchBytes; }

@@ -8,43 +8,13 @@
 #include <cooperative_groups.h>
 #include <math_constants.h>
 
-#include "cp_common.cuh"
+#include "score_common.cuh"
 
 namespace cp {
 namespace {
 
 constexpr int kThreads = 512;
 constexpr int kWarps = kThreads / 32;
-
-template <typename T> __device__ __forceinline__ double to_f64(T x);
-template <> __device__ __forceinline__ double to_f64<float>(float x) { return double(x); }
-template <> __device__ __forceinline__ double to_f64<__nv_bfloat16>(__nv_bfloat16 x) { return double(__bfloat162float(x)); }
-template <> __device__ __forceinline__ double to_f64<__half>(__half x) { return double(__half2float(x)); }
-
-// ln(1 + e^-x), x >= 0, from piecewise degree-11 polynomials on intervals of width 1/2 (absolute error 1e-15;
-// the table and how it is made: gen_softplus_table.py).  The library exp + log pair costs several hundred fp64
-// instructions and this function runs once or twice for every element of the score map.
-constexpr int kSpIntervals = 80, kSpCoef = 12, kSpStride = 13;   // stride 13: rows of different intervals hit different banks
-__device__ const double kSoftplusTable[kSpIntervals * kSpCoef] = {
-#include "softplus_table.inc"
-};
-__device__ __forceinline__ double softplus_neg(double x, const double* tab) {
-  if (!(x < 40.0)) return 0.0;              // e^-40 = 4e-18: below the rounding of whatever it is added to
-  const int i = int(x * 2.0);
-  const double t = (x - (0.5 * i + 0.25)) * 4.0;
-  const double* c = tab + i * kSpStride;
-  double p = c[kSpCoef - 1];
-#pragma unroll
-  for (int k = kSpCoef - 2; k >= 0; --k) p = fma(p, t, c[k]);
-  return p;
-}
-// ln(e^a + e^b) = max + ln(1 + e^-(max - min))
-__device__ __forceinline__ double logaddexp(double a, double b, const double* tab) {
-  const double hi = fmax(a, b), lo = fmin(a, b);
-  const double x = hi - lo;                 // >= 0 (+inf when one term is -inf), or NaN when both are -inf
-  if (!(x >= 0.0)) return hi;
-  return hi + softplus_neg(x, tab);
-}
 
 // Shared memory: logits lg[U][4][nb] (fp64) for the nb key blocks this CTA owns, plus an fp32 copy that
 // the log-sum-exp uses as a filter.  When the 4*U*n2 logits of a row group do not fit one CTA's shared
@@ -55,7 +25,7 @@ __global__ void __launch_bounds__(kThreads)
 score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __restrict__ Kmax,
              const T* __restrict__ Kmin, const double* __restrict__ S_prev, double* __restrict__ S_out,
              int Hq, int g, int n1, int n2, int seg, int blk, double est_scale, double ln_alpha,
-             double ln_1m_alpha, int fuse, int mask_first, int CL, int nb) {
+             double ln_1m_alpha, int fuse, int mask_first, int CL, int nb, double* __restrict__ stats_out) {
   extern __shared__ double smem[];
   double* lg = smem;                                // [U][4][nb]
   float* lf = reinterpret_cast<float*>(smem + 4 * U * nb);   // the same logits rounded to fp32: a cheap filter for the log-sum-exp
@@ -254,10 +224,13 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
   }
   __syncthreads();
 
+  // stats_out given: this launch only produces the four log-sum-exps of every (head, segment) row
+  if (stats_out != nullptr && rank == 0 && tid < 4 * U) stats_out[unit_of(tid >> 2) * 4 + (tid & 3)] = stat[tid];
+
   // combine (lines 11-12), mask (13), fusion (14) over this CTA's blocks of the U rows
   const double ln2 = 0.693147180559945309417232121458;
 #pragma unroll 1
-  for (int u = 0; u < U; ++u) {
+  for (int u = 0; u < (stats_out != nullptr ? 0 : U); ++u) {
     const double* l = lg + u * 4 * nb;
     const double st1 = stat[u * 4 + 0], st2 = stat[u * 4 + 1], st3 = stat[u * 4 + 2], st4 = stat[u * 4 + 3];
     const size_t out_row = unit_of(u) * n2 + b_lo;
@@ -285,7 +258,7 @@ score_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __
 
 template <typename T, int D, int U>
 int launch_u(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
-             double est_scale, double alpha, int fuse, int mask_first, int CL, int nb, cudaStream_t st) {
+             double est_scale, double alpha, int fuse, int mask_first, int CL, int nb, double* stats_out, cudaStream_t st) {
   const size_t smem = (sizeof(double) + sizeof(float)) * (4 * size_t(U) * nb);   // fp64 logits + their fp32 copies
   auto kern = score_kernel<T, D, U>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)) != cudaSuccess)
@@ -305,13 +278,13 @@ int launch_u(const Dims& m, const char* ws, const WsLayout& w, const double* S_p
   const cudaError_t e = cudaLaunchKernelEx(
       &cfg, kern, reinterpret_cast<const T*>(ws + w.qmax), reinterpret_cast<const T*>(ws + w.qmin),
       reinterpret_cast<const T*>(ws + w.kmax), reinterpret_cast<const T*>(ws + w.kmin), S_prev, S_out,
-      m.Hq, m.g, m.n1, m.n2, m.seg, m.blk, est_scale, log(alpha), log1p(-alpha), fuse, mask_first, CL, nb);
+      m.Hq, m.g, m.n1, m.n2, m.seg, m.blk, est_scale, log(alpha), log1p(-alpha), fuse, mask_first, CL, nb, stats_out);
   return e == cudaSuccess ? check_launch() : CP_ERR_CUDA;
 }
 
 template <typename T, int D>
 int launch_t(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
-             double est_scale, double alpha, int fuse, int mask_first, cudaStream_t st) {
+             double est_scale, double alpha, int fuse, int mask_first, double* stats_out, cudaStream_t st) {
   // as many heads per CTA as divide the group (the fp64 MMA has 8 rows = 4 heads x 2 representatives);
   // key blocks are split over a cluster of 1, 2, 4 or 8 CTAs until the logits fit ~200 KB per CTA
   const size_t budget = 200 * 1024;
@@ -319,30 +292,32 @@ int launch_t(const Dims& m, const char* ws, const WsLayout& w, const double* S_p
   for (int CL = 1; CL <= 8; CL *= 2) {
     const int nb = (((m.n2 + CL - 1) / CL) + 7) & ~7;
     if ((sizeof(double) + sizeof(float)) * 4 * size_t(U) * nb > budget) continue;
-    if (U == 4) return launch_u<T, D, 4>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
-    if (U == 2) return launch_u<T, D, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
-    return launch_u<T, D, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, st);
+    if (U == 4) return launch_u<T, D, 4>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, stats_out, st);
+    if (U == 2) return launch_u<T, D, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, stats_out, st);
+    return launch_u<T, D, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, mask_first, CL, nb, stats_out, st);
   }
   return CP_ERR_UNSUPPORTED;
 }
 
 }  // namespace
 
-int launch_score(const cp_params& p, const Dims& m, const char* ws, const double* S_prev,
-                 double* S_out, cudaStream_t st) {
+// The general kernel: any dtype, head_dim 64 or 128.  With stats_out it only writes the four log-sum-exps
+// of every (head, segment) row, [B,Hq,n1,4], and leaves S_out alone.
+int launch_score_generic(const cp_params& p, const Dims& m, const char* ws, const double* S_prev,
+                         double* S_out, double* stats_out, cudaStream_t st) {
   const WsLayout w = ws_layout(m);
   const int fuse = (S_prev != nullptr && p.alpha != 1.0f) ? 1 : 0;
   const int mask_first = (p.flags & CP_FLAG_MASK_BEFORE_SOFTMAX) ? 1 : 0;
   const double es = double(p.est_scale), al = double(p.alpha);
   if (p.dtype == CP_BF16) {
-    if (m.d == 128) return launch_t<__nv_bfloat16, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
-    if (m.d == 64) return launch_t<__nv_bfloat16, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
+    if (m.d == 128) return launch_t<__nv_bfloat16, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, stats_out, st);
+    if (m.d == 64) return launch_t<__nv_bfloat16, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, stats_out, st);
   } else if (p.dtype == CP_F16) {
-    if (m.d == 128) return launch_t<__half, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
-    if (m.d == 64) return launch_t<__half, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
+    if (m.d == 128) return launch_t<__half, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, stats_out, st);
+    if (m.d == 64) return launch_t<__half, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, stats_out, st);
   } else {
-    if (m.d == 128) return launch_t<float, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
-    if (m.d == 64) return launch_t<float, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, st);
+    if (m.d == 128) return launch_t<float, 128>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, stats_out, st);
+    if (m.d == 64) return launch_t<float, 64>(m, ws, w, S_prev, S_out, es, al, fuse, mask_first, stats_out, st);
   }
   return CP_ERR_UNSUPPORTED;
 }

@@ -52,6 +52,40 @@ template <> struct Vec<float> {
   __device__ static uint32_t mn(uint32_t a, uint32_t b) { return __float_as_uint(fminf(__uint_as_float(a), __uint_as_float(b))); }
 };
 
+// largest magnitude among the elements of a 16-byte vector
+template <typename T> __device__ __forceinline__ float vec_absmax(const uint4& a);
+template <> __device__ __forceinline__ float vec_absmax<float>(const uint4& a) {
+  return fmaxf(fmaxf(fabsf(__uint_as_float(a.x)), fabsf(__uint_as_float(a.y))), fmaxf(fabsf(__uint_as_float(a.z)), fabsf(__uint_as_float(a.w))));
+}
+template <> __device__ __forceinline__ float vec_absmax<__nv_bfloat16>(const uint4& a) {
+  const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {   // a bf16 is the upper half of a float
+    m = fmaxf(m, fabsf(__uint_as_float(w[i] << 16)));
+    m = fmaxf(m, fabsf(__uint_as_float(w[i] & 0xffff0000u)));
+  }
+  return m;
+}
+template <> __device__ __forceinline__ float vec_absmax<__half>(const uint4& a) {
+  const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+  float m = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
+    m = fmaxf(m, fmaxf(fabsf(f.x), fabsf(f.y)));
+  }
+  return m;
+}
+// largest magnitude of a group's summaries: every lane holds the group's (max, min) slice of column slot lane % LPR
+template <typename T, int LPR>
+__device__ __forceinline__ float group_absmax(const uint4& mx, const uint4& mn) {
+  float m = fmaxf(vec_absmax<T>(mx), vec_absmax<T>(mn));
+#pragma unroll
+  for (int o = 1; o < LPR; o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  return m;
+}
+
 template <typename T>
 __device__ __forceinline__ void vmax(uint4& a, const uint4& b) {
   a.x = Vec<T>::mx(a.x, b.x); a.y = Vec<T>::mx(a.y, b.y); a.z = Vec<T>::mx(a.z, b.z); a.w = Vec<T>::mx(a.w, b.w);
@@ -72,6 +106,7 @@ struct Side {            // one tensor (Q or K) and where its summaries go
   int64_t sb, sh, st;    // strides in elements
   int H, groups_per_head, G, n;  // heads, groups per head (ceil(n/G)), rows per group (the last may be shorter), tokens
   char *omax, *omin;     // [B,H,groups,d] contiguous
+  float* oabs;           // nullable, [B,H,groups]: largest magnitude in the group's summaries
   long long n_groups;    // B*H*groups_per_head
   long long cta_begin;   // first CTA of this side
   int groups_per_cta;    // kWarps (warp-owned groups) or 1 (CTA-owned group)
@@ -126,13 +161,20 @@ __global__ void __launch_bounds__(kThreads) summarize_kernel(Side q, Side k, int
     for (int m = LPR; m < 32; m <<= 1) { uint4 o = shfl_xor4(mx, m); vmax<T>(mx, o); o = shfl_xor4(mn, m); vmin<T>(mn, o); }
     if (lane < LPR) { red[0][warp][lane] = mx; red[1][warp][lane] = mn; }
     __syncthreads();
-    if (warp == 0 && lane < LPR) {
-      mx = red[0][0][lane]; mn = red[1][0][lane];
+    if (warp == 0) {
+      const int col = lane % LPR;
+      mx = red[0][0][col]; mn = red[1][0][col];
 #pragma unroll
-      for (int w = 1; w < kWarps; ++w) { vmax<T>(mx, red[0][w][lane]); vmin<T>(mn, red[1][w][lane]); }
-      const size_t off = (size_t(grp) * d) * es + lane * 16;
-      *reinterpret_cast<uint4*>(s.omax + off) = mx;
-      *reinterpret_cast<uint4*>(s.omin + off) = mn;
+      for (int w = 1; w < kWarps; ++w) { vmax<T>(mx, red[0][w][col]); vmin<T>(mn, red[1][w][col]); }
+      if (lane < LPR) {
+        const size_t off = (size_t(grp) * d) * es + lane * 16;
+        *reinterpret_cast<uint4*>(s.omax + off) = mx;
+        *reinterpret_cast<uint4*>(s.omin + off) = mn;
+      }
+      if (s.oabs != nullptr) {
+        const float am = group_absmax<T, LPR>(mx, mn);
+        if (lane == 0) s.oabs[grp] = am;
+      }
     }
   } else {
     // each warp owns one group of G <= 128 rows
@@ -152,6 +194,10 @@ __global__ void __launch_bounds__(kThreads) summarize_kernel(Side q, Side k, int
       *reinterpret_cast<uint4*>(s.omax + off) = mx;
       *reinterpret_cast<uint4*>(s.omin + off) = mn;
     }
+    if (s.oabs != nullptr) {
+      const float am = group_absmax<T, LPR>(mx, mn);
+      if (lane == 0) s.oabs[grp] = am;
+    }
   }
 }
 
@@ -169,7 +215,7 @@ int launch_summarize(const cp_params& p, const Dims& m, const void* Q, const voi
   auto mk = [&](const void* base, const int64_t* s, int H, int G, char* omax, char* omin) {
     Side x;
     x.base = static_cast<const char*>(base); x.sb = s[0]; x.sh = s[1]; x.st = s[2];
-    x.H = H; x.G = G; x.n = m.n; x.groups_per_head = (m.n + G - 1) / G; x.omax = omax; x.omin = omin;
+    x.H = H; x.G = G; x.n = m.n; x.groups_per_head = (m.n + G - 1) / G; x.omax = omax; x.omin = omin; x.oabs = nullptr;
     x.n_groups = (long long)m.B * H * x.groups_per_head;
     x.groups_per_cta = G > 128 ? 1 : kWarps;
     x.cta_begin = 0;
@@ -177,6 +223,7 @@ int launch_summarize(const cp_params& p, const Dims& m, const void* Q, const voi
   };
   Side q = mk(Q, p.q_stride, m.Hq, m.seg, ws + w.qmax, ws + w.qmin);
   Side k = mk(K, p.k_stride, m.Hkv, m.blk, ws + w.kmax, ws + w.kmin);
+  k.oabs = reinterpret_cast<float*>(ws + w.kabs);
   const long long q_ctas = (q.n_groups + q.groups_per_cta - 1) / q.groups_per_cta;
   const long long k_ctas = (k.n_groups + k.groups_per_cta - 1) / k.groups_per_cta;
   k.cta_begin = q_ctas;
