@@ -6,7 +6,10 @@ One "step" is one pass of the whole path over one layer's Q/K/V:
 on the 128K-token Llama3-8B-shaped workload (config C4), with inputs resident in HBM.
 Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C4] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C4] [--impl ours|reference] [--shard replicas|heads]
+
+With --gpus N > 1 and no torchrun environment the script starts the N ranks itself
+(python -m torch.distributed.run on 127.0.0.1); under torchrun it is one of the ranks.
 """
 from __future__ import annotations
 
@@ -26,15 +29,22 @@ sys.path.insert(0, ROOT)
 
 from paper_2409_12490_b200 import CONFIGS  # noqa: E402
 from paper_2409_12490_b200.inputs import make_qkv  # noqa: E402
-from paper_2409_12490_b200.sharding import RankInfo, aggregate_time_metric, layer_seed_for_rank, max_over_ranks  # noqa: E402
+from paper_2409_12490_b200.sharding import (RankInfo, aggregate_time_metric, layer_seed_for_rank, max_over_ranks,  # noqa: E402
+                                            shard_heads)
 
 METRIC = "128K prefill-attention ms (estimate+select+sparse attention, one layer)"
-# DRAM bytes (read + write) per launch of the sparse attention kernel, from the ncu captures
-# summarised in profiles/attention_sm100_kernel_C4_counters.md (C4, full size) and
-# profiles/attention_sm100_kernel_C3.md; None for workloads without a capture.
-ATTN_TRAFFIC_BYTES = {"C4": 2.82e9, "C3": 0.640e9}
-# sm__pipe_tensor_cycles_active (% of peak, elapsed) of the same kernel from the same captures
-ATTN_TENSOR_PIPE_PCT = {"C4": 57.7, "C3": 49.1}
+
+
+def load_ncu_counters():
+    """Counters of the sparse attention kernel taken under ncu and kept beside the profile summaries
+    (profiles/attention_counters.json: per workload the DRAM bytes read + written by one launch, the tensor-pipe
+    and XU-pipe active percentages, and the commit and command they were captured with).  They describe the
+    capture, not this run; the run's own figure is the event-timed `achieved`."""
+    path = os.path.join(ROOT, "profiles", "attention_counters.json")
+    if not os.path.exists(path):
+        return {}
+    with open(path) as f:
+        return json.load(f)
 
 
 def load_peaks():
@@ -217,9 +227,27 @@ def workload_config(cfg):
 
 
 # ----------------------------------------------------------------------------- our arm
+def spawn_ranks(n: int) -> int:
+    """Start `n` ranks of this script on this node (one per GPU) and wait for them; rank 0 prints the JSON line."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")                     # the communicator log (transports, NVLS) is kept, in a file:
+    env.setdefault("NCCL_DEBUG_FILE", os.path.join("/tmp", "critiprefill_nccl_%h_%p.log"))   # stdout carries one JSON line only
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
 def run_ours(args, cfg):
     info = RankInfo.from_env()
     rank, world, local = info.rank, info.world, info.local_rank
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s): start bench.py either plainly "
+                         f"(it spawns its own ranks) or under torchrun with --nproc-per-node {args.gpus}")
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -238,13 +266,28 @@ def run_ours(args, cfg):
         dist.barrier()
     cp.load_library()
 
-    # every rank works on its own batch item (same shape, its own seed): weak scaling, no collective.
+    # --shard replicas: every rank works on its own batch item (same shape, its own seed): weak scaling.
+    # --shard heads: ONE problem; rank p owns the KV heads head_shard(Hkv, p, N) and their g query heads and runs
+    # the library on strided views of the full tensors (every (batch, head) is independent in Algorithms 1 and 2):
+    # strong scaling.  Neither mode has a collective on the data path.
     # A stack of L layers cycles through D distinct seeded layer inputs; the criticality scores are
     # carried from layer to layer (Algorithm 1, line 14) through two ping-pong buffers.
+    by_heads = args.shard == "heads" and world > 1
+    full_cfg = cfg
+    shard = shard_heads(cfg, rank, world) if by_heads else None
+    if by_heads:
+        cfg = shard.cfg
     L = args.layers if args.layers else cfg.layers
     D = min(L, args.distinct_layers)
     layers_in = []
     for li in range(D):
+        if by_heads:
+            qf, kf, vf = (t.to(dev) for t in make_qkv(full_cfg, layer=li))               # the same full problem on every rank
+            q, k, v = shard.slice_q(qf), shard.slice_kv(kf), shard.slice_kv(vf)         # views: strides of the full tensors
+            layers_in.append((q, k, v))
+            if li == 0:
+                Q, K, V = q.cpu().contiguous(), k.cpu().contiguous(), v.cpu().contiguous()
+            continue
         q, k, v = make_qkv(cfg, layer=layer_seed_for_rank(li, rank, D))
         if li == 0:
             Q, K, V = q, k, v
@@ -257,7 +300,7 @@ def run_ours(args, cfg):
     S2 = torch.empty_like(S) if L > 1 else None
     idx = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1, cfg.budget_blocks), dtype=torch.int32, device=dev)
     cnt = torch.empty((cfg.batch, cfg.n_q_heads, cfg.n1), dtype=torch.int32, device=dev)
-    O = torch.empty_like(dQ)
+    O = torch.empty(dQ.shape, dtype=dQ.dtype, device=dev)
     hO = torch.empty_like(hQ).pin_memory()
     torch.cuda.synchronize()
 
@@ -314,13 +357,13 @@ def run_ours(args, cfg):
     sel_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     att_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     total_ms, est_ms, sel_ms, att_ms = max_over_ranks([total_ms, est_ms, sel_ms, att_ms], dist, dev)
-    agg = aggregate_time_metric(total_ms / args.steps / L, world)      # per layer pass
+    agg = aggregate_time_metric(total_ms / args.steps / L, world, replicas=not by_heads)      # per layer pass
     ms_per_step = agg["ms_per_step"]
 
     # dense baseline of the same library (the denominator of the speed-up)
     dense_ms = None
     if not args.no_dense:
-        Od = torch.empty_like(dQ)
+        Od = torch.empty(dQ.shape, dtype=dQ.dtype, device=dev)
         cp.dense_attention(prob, dQ, dK, dV, ws, O=Od)
         torch.cuda.synchronize()
         d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -383,23 +426,29 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
         att_ms, est_ms, sel_ms = a0.elapsed_time(a1) / 5, None, None
     achieved = fl["executed"] / (att_ms * 1e-3) / 1e12
+    ncu = load_ncu_counters().get(cfg.name, {})
     roofline = {"bound": "tensor", "kernel": "attention_sm100_kernel (critiprefill_attention)",
                 "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_tflops"], "peak_source": f"{peaks['source']} (burst)",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
-                "flops_per_launch": fl["executed"], "traffic": ATTN_TRAFFIC_BYTES.get(cfg.name),
-                "tensor_pipe_active_pct_ncu": ATTN_TENSOR_PIPE_PCT.get(cfg.name),
-                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, ncu)"}
+                "flops_per_launch": fl["executed"], "traffic": ncu.get("dram_bytes_per_launch"),
+                "tensor_pipe_active_pct_ncu": ncu.get("tensor_pipe_active_pct"),
+                "ncu_capture": {k: ncu.get(k) for k in ("commit", "captured", "command")} if ncu else None,
+                "traffic_unit": "bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, from the ncu capture named in "
+                                "ncu_capture; not measured in this run)"}
     summary_bytes = (dQ.numel() + dK.numel()) * dQ.element_size()
     out = {
         "metric": METRIC, "value": ms_per_step, "unit": "ms", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": workload_config(cfg),
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False,
+        "scaling": "strong" if by_heads else "weak",
+        "sharding": ("heads: one layer, each rank owns Hkv/N KV heads and their query heads (no collective on the path)" if by_heads
+                     else "replicas: one layer per rank (no collective on the path)") if world > 1 else "single GPU",
+        "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": workload_config(full_cfg),
         "breakdown_ms": {"estimate": est_ms, "select": sel_ms, "attention": att_ms},
         "dense_ms": dense_ms,
         "speedup_vs_dense": (dense_ms / ms_per_step) if dense_ms else None,
-        "dense_equiv_tflops": fl["dense"] / (ms_per_step * 1e-3) / 1e12,
+        "dense_equiv_tflops": flop_counts(full_cfg)["dense"] * (1 if by_heads else world) / (ms_per_step * 1e-3) / 1e12,
         "dense_kernel_tflops": (fl["dense"] / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
         "estimate_gbs": (summary_bytes / (est_ms * 1e-3) / 1e9) if est_ms else None,
         "layer_passes_per_s": agg["layer_passes_per_s"],
@@ -563,10 +612,14 @@ def main():
                     help="layer fusion on/off over a stack of --layers seeded layers (quality diagnostic) instead of the bench line")
     ap.add_argument("--overlap", action="store_true",
                     help="token-wise critical-set overlap between neighbouring queries (Eq. 3; quality diagnostic) instead of the bench line")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="with --gpus N > 1: N independent layers (weak scaling) or one layer split by KV head group (strong scaling)")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
+    if args.impl == "ours" and args.gpus > 1 and "RANK" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     if args.impl == "reference":
         run_reference(args, cfg)
     elif args.sweep:
