@@ -13,19 +13,50 @@ than k blocks take all of them (cnt < k, list padded with -1); lists are ascendi
 sequence length that is not a multiple of the segment size the last segment overlaps fewer than r
 blocks and the slots it does not need go to past blocks.
 The selection itself is pinned (tests above); which reading the authors' code takes is parity unpinned.
+
+Variants the paper's text does not fix (readings of this build, each pinned against brute force and against the
+plain selection as their special case):
+  * shared lists per KV group (``group``): the g query heads that share a KV head use ONE list per segment, taken
+    from the element-wise maximum of their scores (the maximum of the probabilities S, i.e. of ln S) -- a block
+    that is critical for any head of the group is kept for all of them;
+  * forced sink / local blocks (``n_sink``, ``n_local``): the first n_sink blocks of the sequence and the n_local
+    blocks right before the segment are always kept, like the diagonal blocks, and count against the budget;
+    n_sink + n_local <= k - r is required, so they always fit.
 """
 from __future__ import annotations
 
 import numpy as np
 
 
-def select(S: np.ndarray, segment_size: int, block_size: int, budget_blocks: int):
-    """S: ln-scores [B,Hq,n1,n2] -> (idx int32 [B,Hq,n1,k], cnt int32 [B,Hq,n1])."""
+def pool_group_scores(S: np.ndarray, group: int) -> np.ndarray:
+    """Element-wise maximum of ln S over the `group` consecutive query heads that share a KV head, written back to
+    every head of the group: [B,Hq,n1,n2] -> [B,Hq,n1,n2]."""
     S = np.asarray(S, dtype=np.float64)
+    B, H, n1, n2 = S.shape
+    assert H % group == 0
+    out = np.empty_like(S)
+    for b in range(B):
+        for kv in range(H // group):
+            pooled = S[b, kv * group]
+            for h in range(kv * group + 1, (kv + 1) * group):
+                pooled = np.maximum(pooled, S[b, h])
+            for h in range(kv * group, (kv + 1) * group):
+                out[b, h] = pooled
+    return out
+
+
+def select(S: np.ndarray, segment_size: int, block_size: int, budget_blocks: int, *, group: int = 1,
+           n_sink: int = 0, n_local: int = 0):
+    """S: ln-scores [B,Hq,n1,n2] -> (idx int32 [B,Hq,n1,k], cnt int32 [B,Hq,n1]).
+    group > 1: one list per KV group (see the module text); n_sink / n_local: forced past blocks."""
+    S = np.asarray(S, dtype=np.float64)
+    if group > 1:
+        S = pool_group_scores(S, group)
     B, H, n1, n2 = S.shape
     r = segment_size // block_size
     k = budget_blocks
     assert segment_size % block_size == 0 and r <= k
+    assert n_sink >= 0 and n_local >= 0 and n_sink + n_local <= k - r
     idx = np.full((B, H, n1, k), -1, dtype=np.int32)
     cnt = np.zeros((B, H, n1), dtype=np.int32)
     for b in range(B):
@@ -37,7 +68,9 @@ def select(S: np.ndarray, segment_size: int, block_size: int, budget_blocks: int
                 if past <= m:
                     chosen = list(range(past))
                 else:
-                    row = S[b, h, j, :past]
+                    row = S[b, h, j, :past].copy()
+                    forced = [x for x in range(past) if x < n_sink or x >= past - n_local]
+                    row[forced] = np.inf                   # forced blocks come before every scored block
                     # descending by (score, index): stable ascending argsort of the reversed row
                     order = np.argsort(-row[::-1], kind="stable")
                     chosen = sorted(int(past - 1 - o) for o in order[:m])

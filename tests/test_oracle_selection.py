@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from oracle.selection import select
+from oracle.selection import pool_group_scores, select
 
 
 def scores(n1, n2, seed, ties=False):
@@ -81,3 +81,64 @@ def test_short_last_segment(n, seg, blk, k):
             want = sorted(ranked[:k - len(diag)] + diag)
             assert idx[0, h, j, :cnt[0, h, j]].tolist() == want
             assert cnt[0, h, j] == min(k, len(past) + len(diag))
+
+
+def test_group_pooling_is_the_elementwise_maximum_and_group_one_changes_nothing():
+    rng = np.random.default_rng(8)
+    S = rng.standard_normal((2, 6, 5, 20))
+    S[:, :, :, 15:] = -np.inf
+    P = pool_group_scores(S, 3)
+    for b in range(2):
+        for h in range(6):
+            for j in range(5):
+                for x in range(20):
+                    kv = h // 3
+                    assert P[b, h, j, x] == max(S[b, kv * 3 + u, j, x] for u in range(3))
+    assert np.array_equal(pool_group_scores(S, 1), S)
+    seg, blk, k = 8, 2, 6
+    S = scores(12, 48, 9)
+    a = select(S, seg, blk, k)
+    b = select(S, seg, blk, k, group=1)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("ties", [False, True])
+def test_shared_group_lists_against_brute_force(ties):
+    seg, blk, k, n, g = 8, 2, 7, 96, 2
+    n1, n2, r = n // seg, n // blk, seg // blk
+    rng = np.random.default_rng(10)
+    S = rng.standard_normal((1, 4, n1, n2))
+    if ties:
+        S = np.round(S * 2) / 2
+    idx, cnt = select(S, seg, blk, k, group=g)
+    for kv in range(2):
+        for j in range(n1):
+            past = list(range(j * r))
+            pooled = {x: max(S[0, kv * g + u, j, x] for u in range(g)) for x in past}
+            ranked = sorted(past, key=lambda x: (pooled[x], x), reverse=True)
+            want = sorted(ranked[:k - r] + list(range(j * r, (j + 1) * r)))
+            for u in range(g):                                   # every head of the group gets the same list
+                assert idx[0, kv * g + u, j, :cnt[0, kv * g + u, j]].tolist() == want
+
+
+@pytest.mark.parametrize("n_sink,n_local,ties", [(1, 0, False), (0, 2, False), (2, 1, True), (1, 1, True)])
+def test_forced_sink_and_local_blocks_against_brute_force(n_sink, n_local, ties):
+    seg, blk, k, n = 8, 2, 9, 128
+    n1, n2, r = n // seg, n // blk, seg // blk
+    S = scores(n1, n2, 11, ties)
+    idx, cnt = select(S, seg, blk, k, n_sink=n_sink, n_local=n_local)
+    plain = select(S, seg, blk, k)
+    for h in range(2):
+        for j in range(n1):
+            past = list(range(j * r))
+            forced = [x for x in past if x < n_sink or x >= j * r - n_local]
+            free = [x for x in past if x not in forced]
+            ranked = sorted(free, key=lambda x: (S[0, h, j, x], x), reverse=True)
+            m = k - r
+            want = sorted(past) if len(past) <= m else sorted(forced + ranked[:m - len(forced)])
+            want = want + list(range(j * r, (j + 1) * r))
+            got = idx[0, h, j, :cnt[0, h, j]].tolist()
+            assert got == want and set(forced) <= set(got)
+            assert cnt[0, h, j] == plain[1][0, h, j]            # forced blocks count against the same budget
+    z = select(S, seg, blk, k, n_sink=0, n_local=0)
+    assert np.array_equal(z[0], plain[0])
