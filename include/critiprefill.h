@@ -61,9 +61,12 @@ typedef enum { CP_BF16 = 0, CP_F32 = 1, CP_F16 = 2 } cp_dtype;   /* fp16 is the 
 enum {
   CP_FLAG_MASK_BEFORE_SOFTMAX = 1, /* estimate: normalise each score map over visible blocks only */
   CP_FLAG_FORCE_SIMT = 2,          /* attention: use the SIMT kernel even where tensor cores apply */
-  CP_FLAG_TEST_WITHHOLD_V = 4      /* test hook for the bounded waits of the tensor-core kernel: V tiles are
+  CP_FLAG_TEST_WITHHOLD_V = 4,     /* test hook for the bounded waits of the tensor-core kernel: V tiles are
                                       never loaded, so a pipeline wait expires after about 2 s, the kernel
                                       drains and the status block reads CP_ERR_TIMEOUT (outputs invalid) */
+  CP_FLAG_SHARED_GROUP_LISTS = 8   /* select: one list per KV group instead of one per query head -- the g query
+                                      heads of a KV head all receive the list selected from the element-wise
+                                      maximum of their scores (a variant; the paper describes a single head) */
 };
 
 typedef struct {
@@ -76,7 +79,10 @@ typedef struct {
   float sm_scale;  /* attention logit scale, 1/sqrt(head_dim) in Eq. 2 / Algorithm 2 line 10 */
   float alpha;     /* layer-fusion weight of the current layer (Algorithm 1 line 14; 0.25 in
                       Section 3.1.3), in [0, 1] (else CP_ERR_SHAPE); ignored when S_prev is NULL */
-  int32_t reserved;
+  int32_t forced_blocks; /* select: n_sink | (n_local << 16), normally 0.  The first n_sink blocks of the sequence
+                            and the n_local blocks right before each segment are always listed, like the diagonal
+                            blocks, and count against k; requires n_sink + n_local <= k - r (else CP_ERR_SHAPE).
+                            A variant: the paper fixes no sink or local blocks */
 } cp_params;
 
 /* Bytes of scratch (`ws`) the calls below need for these parameters; the same buffer serves
@@ -133,7 +139,9 @@ size_t critiprefill_static_scratch_bytes(void);
  *             segment j ([j*r, min(n2,(j+1)*r)); r_j = r except in a short last segment) are
  *             always present and count against k; the other k-r_j entries are the
  *             strictly-past blocks with the largest S[j,b], ties to the larger b; entries
- *             beyond cnt are -1
+ *             beyond cnt are -1.  With CP_FLAG_SHARED_GROUP_LISTS the score of a block is the
+ *             largest over the g query heads of the KV group and those heads share the list;
+ *             forced_blocks adds always-kept sink / local blocks (see cp_params)
  *   cnt  out  device, [B,Hq,n1] int32 = min(k, number of blocks visible to segment j)
  * Exact (comparisons only). */
 int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws,

@@ -21,6 +21,7 @@ CP_BF16, CP_F32, CP_F16 = 0, 1, 2
 FLAG_MASK_BEFORE_SOFTMAX = 1
 FLAG_FORCE_SIMT = 2
 FLAG_TEST_WITHHOLD_V = 4
+FLAG_SHARED_GROUP_LISTS = 8
 
 EXPORTS = (
     "critiprefill_workspace_bytes", "critiprefill_estimate", "critiprefill_select",
@@ -39,7 +40,7 @@ class CpParams(ctypes.Structure):
         ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3),
         ("v_stride", ctypes.c_int64 * 3), ("o_stride", ctypes.c_int64 * 3),
         ("est_scale", ctypes.c_float), ("sm_scale", ctypes.c_float), ("alpha", ctypes.c_float),
-        ("reserved", ctypes.c_int32),
+        ("forced_blocks", ctypes.c_int32),
     ]
 
 
@@ -117,6 +118,8 @@ class Problem:
     sm_scale: float | None = None
     alpha: float = 0.25
     flags: int = 0
+    n_sink: int = 0      # always-kept first blocks of the sequence (variant; counts against the budget)
+    n_local: int = 0     # always-kept blocks right before each segment (variant; counts against the budget)
 
     @classmethod
     def from_config(cls, cfg, **kw) -> "Problem":
@@ -151,6 +154,7 @@ class Problem:
         p.est_scale = self.est_scale
         p.sm_scale = self.sm_scale if self.sm_scale is not None else 1.0 / math.sqrt(self.head_dim)
         p.alpha = self.alpha
+        p.forced_blocks = self.n_sink | (self.n_local << 16)
         return p
 
 

@@ -15,6 +15,7 @@ int validate(const cp_params* p, Dims* out) {
   if (p->segment_size % p->block_size) return CP_ERR_SHAPE;
   Dims m = make_dims(*p);
   if (m.k < m.r) return CP_ERR_SHAPE;
+  if (p->forced_blocks < 0 || (p->forced_blocks & 0xffff) + ((p->forced_blocks >> 16) & 0xffff) > m.k - m.r) return CP_ERR_SHAPE;
   if (m.d != 64 && m.d != 128) return CP_ERR_UNSUPPORTED;
   const int64_t align = 16 / m.es;
   const int64_t* strides[4] = {p->q_stride, p->k_stride, p->v_stride, p->o_stride};

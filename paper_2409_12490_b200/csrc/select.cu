@@ -42,21 +42,25 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int lane, int warp, i
 
 // KPT = keys per thread; thread t owns the KPT consecutive blocks [t*KPT, (t+1)*KPT), so the ordered
 // compaction at the end is two block-wide scans instead of a barrier-separated step per key slot.
+// `pool` > 1: one CTA per (batch, KV head, segment); the key of a block is the largest of the pool's `pool`
+// consecutive query heads' scores, and the one list is written for each of them.  n_sink / n_local: the first
+// n_sink blocks and the n_local blocks right before the segment get the largest possible key, so they are taken
+// before any scored block (the host has checked that they fit into the k - r free slots).
 template <int KPT>
 __global__ void __launch_bounds__(kThreads)
 select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* __restrict__ cnt,
-              int n1, int n2, int r, int k) {
+              int n1, int n2, int r, int k, int pool, int n_sink, int n_local) {
   __shared__ unsigned int hist[256];
   __shared__ int warp_sum[kWarps];
   __shared__ unsigned long long prefix_sh;
   __shared__ int remaining_sh, bin_count_sh;
   __shared__ int warp_tot[kWarps];
 
-  const int unit = blockIdx.x;
-  const int j = unit % n1;
+  // CTA -> (batch * heads / pool + pooled head, segment); its first query head's unit is `unit`
+  const int j = blockIdx.x % n1;
+  const int unit = (blockIdx.x / n1) * pool * n1 + j;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const double* row = S + size_t(unit) * n2;
-  int32_t* out = idx + size_t(unit) * k;
   const int past = j * r;
   const int rj = min(n2, past + r) - past;   // diagonal blocks of this segment (fewer in a short last segment)
   const int m = k - rj;
@@ -64,22 +68,40 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
   if (past <= m) {
     // every visible block fits in the budget
     const int c = past + rj;
-    for (int i = tid; i < k; i += kThreads) out[i] = i < c ? i : -1;
-    if (tid == 0) cnt[unit] = c;
+    for (int u = 0; u < pool; ++u) {
+      int32_t* out = idx + (size_t(unit) + size_t(u) * n1) * k;
+      for (int i = tid; i < k; i += kThreads) out[i] = i < c ? i : -1;
+      if (tid == 0) cnt[unit + u * n1] = c;
+    }
     return;
   }
 
   if (m == 0) {
     // the budget holds the diagonal blocks only
-    for (int i = tid; i < k; i += kThreads) out[i] = i < rj ? past + i : -1;
-    if (tid == 0) cnt[unit] = rj;
+    for (int u = 0; u < pool; ++u) {
+      int32_t* out = idx + (size_t(unit) + size_t(u) * n1) * k;
+      for (int i = tid; i < k; i += kThreads) out[i] = i < rj ? past + i : -1;
+      if (tid == 0) cnt[unit + u * n1] = rj;
+    }
     return;
   }
 
   const int b0 = tid * KPT;                  // first block owned by this thread
   unsigned long long key[KPT];
 #pragma unroll
-  for (int s = 0; s < KPT; ++s) key[s] = b0 + s < past ? ordered_key(__ldg(row + b0 + s)) : 0ull;
+  for (int s = 0; s < KPT; ++s) {
+    const int bb = b0 + s;
+    unsigned long long kk = 0ull;
+    if (bb < past) {
+      if (bb < n_sink || bb >= past - n_local) {
+        kk = ~0ull;                          // forced block
+      } else {
+        kk = ordered_key(__ldg(row + bb));
+        for (int u = 1; u < pool; ++u) kk = max(kk, ordered_key(__ldg(row + size_t(u) * n1 * n2 + bb)));
+      }
+    }
+    key[s] = kk;
+  }
   hist[tid] = 0;
   __syncthreads();
 
@@ -145,33 +167,38 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
 
   // ---- ordered compaction: blocks are owned in index order, so positions are an exclusive scan ----
   int total_take;
-  int pos = block_exclusive_scan(n_take, lane, warp, warp_tot, &total_take);
+  const int pos0 = block_exclusive_scan(n_take, lane, warp, warp_tot, &total_take);
+  for (int u = 0; u < pool; ++u) {           // the same list for every head of the pool
+    int32_t* out = idx + (size_t(unit) + size_t(u) * n1) * k;
+    int pos = pos0;
 #pragma unroll
-  for (int s = 0, e = eq_before; s < KPT; ++s) {
-    if (b0 + s >= past) break;
-    bool take;
-    if (all_of_bin) take = key[s] >= thr;
-    else if (key[s] == thr) { take = e >= eq_skip; ++e; }
-    else take = key[s] > thr;
-    if (take) { if (pos < m) out[pos] = b0 + s; ++pos; }
+    for (int s = 0, e = eq_before; s < KPT; ++s) {
+      if (b0 + s >= past) break;
+      bool take;
+      if (all_of_bin) take = key[s] >= thr;
+      else if (key[s] == thr) { take = e >= eq_skip; ++e; }
+      else take = key[s] > thr;
+      if (take) { if (pos < m) out[pos] = b0 + s; ++pos; }
+    }
+    for (int i = tid; i < rj; i += kThreads) out[m + i] = past + i;   // diagonal blocks
+    if (tid == 0) cnt[unit + u * n1] = k;
   }
-  for (int i = tid; i < rj; i += kThreads) out[m + i] = past + i;   // diagonal blocks
-  if (tid == 0) cnt[unit] = k;
 }
 
 }  // namespace
 
 int launch_select(const cp_params& p, const Dims& m, const double* S, int32_t* idx, int32_t* cnt,
                   cudaStream_t st) {
-  (void)p;
-  const long long units = (long long)m.B * m.Hq * m.n1;
+  const int pool = (p.flags & CP_FLAG_SHARED_GROUP_LISTS) ? m.g : 1;
+  const int n_sink = p.forced_blocks & 0xffff, n_local = (p.forced_blocks >> 16) & 0xffff;
+  const long long units = (long long)m.B * (m.Hq / pool) * m.n1;
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
   const int kpt = (m.n2 + kThreads - 1) / kThreads;
   const unsigned grid = unsigned(units);
-  if (kpt <= 4) select_kernel<4><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k);
-  else if (kpt <= 8) select_kernel<8><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k);
-  else if (kpt <= 16) select_kernel<16><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k);
-  else if (kpt <= 32) select_kernel<32><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k);
+  if (kpt <= 4) select_kernel<4><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
+  else if (kpt <= 8) select_kernel<8><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
+  else if (kpt <= 16) select_kernel<16><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
+  else if (kpt <= 32) select_kernel<32><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
   else return CP_ERR_UNSUPPORTED;
   return check_launch();
 }

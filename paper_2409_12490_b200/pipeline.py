@@ -26,7 +26,7 @@ class HostPipelinedLayer:
         g = prob.n_q_heads // prob.n_kv_heads
         self.g = g
         self.sub = cp.Problem(1, g, 1, prob.seq_len, prob.head_dim, prob.segment_size, prob.block_size,
-                              prob.budget_blocks, prob.dtype, prob.est_scale, prob.sm_scale, prob.alpha, prob.flags)
+                              prob.budget_blocks, prob.dtype, prob.est_scale, prob.sm_scale, prob.alpha, prob.flags, prob.n_sink, prob.n_local)
         n, d = prob.seq_len, prob.head_dim
         self.dQ = torch.empty((1, prob.n_q_heads, n, d), dtype=prob.dtype, device=self.dev)
         self.dK = torch.empty((1, prob.n_kv_heads, n, d), dtype=prob.dtype, device=self.dev)
@@ -37,7 +37,7 @@ class HostPipelinedLayer:
         self.idx = torch.empty((1, g, self.sub.n1, prob.budget_blocks), dtype=torch.int32, device=self.dev)
         self.cnt = torch.empty((1, g, self.sub.n1), dtype=torch.int32, device=self.dev)
         self.head = cp.Problem(1, 1, 1, prob.seq_len, prob.head_dim, prob.segment_size, prob.block_size,
-                               prob.budget_blocks, prob.dtype, prob.est_scale, prob.sm_scale, prob.alpha, prob.flags)
+                               prob.budget_blocks, prob.dtype, prob.est_scale, prob.sm_scale, prob.alpha, prob.flags, prob.n_sink, prob.n_local)
         self.s_in, self.s_run, self.s_out = (torch.cuda.Stream(self.dev) for _ in range(3))
         self.ev_in = [torch.cuda.Event() for _ in range(prob.n_kv_heads)]
         self.ev_run = [torch.cuda.Event() for _ in range(prob.n_q_heads)]

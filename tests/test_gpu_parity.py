@@ -170,6 +170,38 @@ def test_select_with_ties_matches_oracle():
     assert np.array_equal(idx.cpu().numpy(), idx_ref) and np.array_equal(cnt.cpu().numpy(), cnt_ref)
 
 
+@pytest.mark.parametrize("n_sink,n_local,shared", [(0, 0, True), (1, 2, False), (2, 1, True)])
+def test_selection_variants_match_oracle(n_sink, n_local, shared):
+    """One list per KV group (score = maximum over the group's heads) and forced sink / local blocks, alone and
+    together; then attention on the GPU's lists against the oracle on the same lists."""
+    cfg = SMALL_BF16.with_(block_size=32, budget_tokens=512)          # r = 8, k = 16: 8 free slots
+    Q, K, V = make_qkv(cfg)
+    g = cfg.n_q_heads // cfg.n_kv_heads
+    flags = cp.FLAG_SHARED_GROUP_LISTS if shared else 0
+    prob = problem(cfg, flags=flags, n_sink=n_sink, n_local=n_local)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    S = cp.estimate(prob, Qd, Kd, ws)
+    idx, cnt = cp.select(prob, S, ws)
+    S_ref = oracle_scores(cfg, Q, K)
+    compare_scores(S, S_ref)
+    idx_ref, cnt_ref = oracle.select(S_ref, cfg.segment_size, cfg.block_size, cfg.budget_blocks, group=g if shared else 1,
+                                     n_sink=n_sink, n_local=n_local)
+    assert np.array_equal(idx.cpu().numpy(), idx_ref) and np.array_equal(cnt.cpu().numpy(), cnt_ref)
+    if shared:
+        assert torch.equal(idx[:, 0::2], idx[:, 1::2])                  # g = 2: both heads of a group share the list
+    O = cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws)
+    assert cp.device_status(ws) == 0
+    O_ref, _ = oracle.sparse_attention(Q, K, V, idx_ref, cnt_ref, cfg.segment_size, cfg.block_size, f32(1.0 / np.sqrt(cfg.head_dim)))
+    assert_attention_close(O, O_ref)
+    # heavy ties on top of the variants
+    rng = np.random.default_rng(1)
+    St = np.round(rng.standard_normal(S_ref.shape) * 2) / 2
+    it, ct = cp.select(prob, torch.from_numpy(St).cuda(), ws)
+    ir, cr = oracle.select(St, cfg.segment_size, cfg.block_size, cfg.budget_blocks, group=g if shared else 1, n_sink=n_sink, n_local=n_local)
+    assert np.array_equal(it.cpu().numpy(), ir) and np.array_equal(ct.cpu().numpy(), cr)
+
+
 def test_bad_list_sets_bounds_status_without_faulting():
     cfg = SMALL_BF16
     Q, K, V = make_qkv(cfg)
@@ -198,6 +230,10 @@ def test_host_side_argument_errors():
         cp.workspace_bytes(bad)
     assert e.value.status == 2
     bad = cp.Problem.from_config(cfg.with_(budget_tokens=128))     # budget smaller than one segment
+    with pytest.raises(cp.CritiPrefillError) as e:
+        cp.workspace_bytes(bad)
+    assert e.value.status == 2
+    bad = cp.Problem.from_config(cfg, n_sink=3, n_local=2)         # k - r = 4 free slots cannot hold 5 forced blocks
     with pytest.raises(cp.CritiPrefillError) as e:
         cp.workspace_bytes(bad)
     assert e.value.status == 2
