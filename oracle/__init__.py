@@ -4,6 +4,6 @@ TEST INFRASTRUCTURE ONLY: imported by tests/, by __graft_entry__.smoke() and by
 bench.py's CPU-baseline legs.  The CUDA product path never imports it, and it
 imports nothing from the CUDA package.
 """
-from .estimation import summaries, logits, estimate, causal_block_mask  # noqa: F401
-from .selection import select, pool_group_scores  # noqa: F401
+from .estimation import summaries, logits, estimate, causal_block_mask, decode_estimate  # noqa: F401
+from .selection import select, pool_group_scores, decode_select  # noqa: F401
 from .attention import sparse_attention, dense_attention, sparse_attention_rows, dense_attention_rows  # noqa: F401

@@ -118,3 +118,28 @@ def estimate(Q, K, segment_size: int, block_size: int, *, est_scale: float = 1.0
             ln_a, ln_1ma = np.log(np.float64(alpha)), np.log1p(-np.float64(alpha))
         Lg = _logaddexp(ln_a + Lg, ln_1ma + Lprev)                               # ln(a*S + (1-a)*S')
     return Lg
+
+
+def decode_estimate(q_last, K, block_size: int, *, est_scale: float = 1.0) -> np.ndarray:
+    """Criticality of every key block for the LAST query token (the decoding-phase use of query criticality that
+    Section 2.1 describes: the query of the last token against the cached keys).  Algorithm 1 with the one-token
+    segment {q}: Qmax = Qmin = q, no block lies in the token's future, no previous layer.
+    q_last [B,Hq,d], K [B,Hkv,n,d] -> ln S [B,Hq,n2] fp64.
+
+    Reading (the paper gives no formula for the decoding phase): the segment-wise estimator applied to a segment of
+    one token.  Pins (tests/test_oracle_estimation.py): with block_size = 1 it is the last row of `estimate` run with
+    segment_size = block_size = 1 (Algorithm 1 itself); for any block size, max(softmax(q Kmax^T), softmax(q Kmin^T))
+    written out with loops."""
+    q = _f64(q_last)
+    K = _f64(K)
+    B, Hq, d = q.shape
+    n = K.shape[2]
+    _, _, Kmax, Kmin = summaries(np.zeros((B, Hq, n, d)), K, n, block_size)      # key-block summaries (lines 5-8)
+    qrep = q[:, :, None, :]                                                      # the segment's two representatives coincide
+    L = []
+    for krep in (Kmax, Kmin, Kmax, Kmin):                                        # S1..S4 with Qmax = Qmin
+        l = logits(qrep, krep, est_scale)
+        L.append(l - _logsumexp(l, axis=-1))
+    Lmax = _logaddexp(L[0], L[2]) - LN2
+    Lmin = _logaddexp(L[1], L[3]) - LN2
+    return np.maximum(Lmax, Lmin)[:, :, 0, :]

@@ -78,3 +78,26 @@ def select(S: np.ndarray, segment_size: int, block_size: int, budget_blocks: int
                 cnt[b, h, j] = len(sel)
                 idx[b, h, j, :len(sel)] = sel
     return idx, cnt
+
+
+def decode_select(S: np.ndarray, budget_blocks: int):
+    """Critical blocks of the last query token: S ln-scores [B,Hq,n2] -> (idx int32 [B,Hq,k] ascending, -1 padded;
+    cnt int32 [B,Hq]).  The block that holds the token itself (the last one) is always kept and counts against the
+    budget; the other k-1 slots go to the blocks with the largest score, ties to the larger index."""
+    S = np.asarray(S, dtype=np.float64)
+    B, H, n2 = S.shape
+    k = budget_blocks
+    idx = np.full((B, H, k), -1, dtype=np.int32)
+    cnt = np.zeros((B, H), dtype=np.int32)
+    for b in range(B):
+        for h in range(H):
+            past = n2 - 1
+            if past <= k - 1:
+                chosen = list(range(past))
+            else:
+                order = np.argsort(-S[b, h, :past][::-1], kind="stable")
+                chosen = sorted(int(past - 1 - o) for o in order[:k - 1])
+            sel = chosen + [n2 - 1]
+            cnt[b, h] = len(sel)
+            idx[b, h, :len(sel)] = sel
+    return idx, cnt

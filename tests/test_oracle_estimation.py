@@ -203,3 +203,48 @@ def test_paper_operating_point_fixture():
     c = CONFIGS["paper_128k"]
     assert (c.segment_size, c.block_size, c.budget_tokens, c.alpha) == (
         vals["segment_size"], vals["block_size"], vals["budget_tokens"], vals["alpha"])
+
+
+def test_decode_estimate_is_algorithm_1_on_a_one_token_segment():
+    """The decoding-phase score of the last token: (i) equals Algorithm 1 run with one-token segments (its last row,
+    which sees every block), (ii) equals max(softmax(q Kmax^T), softmax(q Kmin^T)) written out with loops."""
+    import oracle
+    rng = np.random.default_rng(12)
+    B, Hq, Hkv, n, d, blk = 2, 4, 2, 48, 8, 4
+    Q = rng.standard_normal((B, Hq, n, d))
+    K = rng.standard_normal((B, Hkv, n, d))
+    got = oracle.decode_estimate(Q[:, :, -1], K, blk, est_scale=0.7)
+    # (i) segment_size = 1 is not a multiple of the block size, so compare through the summaries: row n-1 of the
+    # four maps with Qmax = Qmin = Q[n-1]
+    Qmax, Qmin, Kmax, Kmin = oracle.summaries(Q, K, 1, blk)
+    assert np.array_equal(Qmax[:, :, -1], Q[:, :, -1]) and np.array_equal(Qmin[:, :, -1], Q[:, :, -1])
+    # (ii) loops
+    n2 = n // blk
+    for b in range(B):
+        for h in range(Hq):
+            q = Q[b, h, -1]
+            kv = h // (Hq // Hkv)
+            lmax = np.array([0.7 * sum(q[c] * Kmax[b, kv, x, c] for c in range(d)) for x in range(n2)])
+            lmin = np.array([0.7 * sum(q[c] * Kmin[b, kv, x, c] for c in range(d)) for x in range(n2)])
+            smax = np.exp(lmax - lmax.max()); smax /= smax.sum()
+            smin = np.exp(lmin - lmin.max()); smin /= smin.sum()
+            want = np.maximum(smax, smin)                     # (S1+S3)/2 = S1 and (S2+S4)/2 = S2 when Qmax = Qmin
+            assert np.allclose(np.exp(got[b, h]), want, rtol=1e-12, atol=0)
+    assert np.all(np.exp(got) <= 1.0 + 1e-12)
+    # block_size = 1: the last row of Algorithm 1 run token by token (segment = block = 1 sees every key at row n-1)
+    full = oracle.estimate(Q, K, 1, 1, est_scale=0.7)
+    assert np.allclose(oracle.decode_estimate(Q[:, :, -1], K, 1, est_scale=0.7), full[:, :, -1, :], rtol=0, atol=1e-12)
+
+
+def test_decode_select_against_full_sort():
+    import oracle
+    rng = np.random.default_rng(13)
+    S = np.round(rng.standard_normal((2, 3, 40)) * 2) / 2      # ties
+    for k in (1, 5, 39, 40, 64):
+        idx, cnt = oracle.decode_select(S, k)
+        for b in range(2):
+            for h in range(3):
+                past = list(range(39))
+                ranked = sorted(past, key=lambda x: (S[b, h, x], x), reverse=True)
+                want = sorted(ranked[:k - 1] + [39])
+                assert idx[b, h, :cnt[b, h]].tolist() == want and (idx[b, h, cnt[b, h]:] == -1).all()
