@@ -147,6 +147,24 @@ size_t critiprefill_static_scratch_bytes(void);
 int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws,
                         size_t ws_bytes, void* cuda_stream);
 
+/* Query criticality of the LAST token, the decoding-phase use that Section 2.1 describes (the query of the last
+ * token against the cached keys).  The paper gives no formula for it; this is Algorithm 1 on a segment that holds
+ * that one token: Qmax = Qmin = q, every block is visible, no layer fusion.
+ *   q_last  in   device, [batch, n_q_heads, head_dim] contiguous, dtype as in p
+ *   K       in   device, layout and strides as in p (seq_len tokens)
+ *   S_out   out  device, [B,Hq,n2] fp64: ln max( softmax_b(q.Kmax_b), softmax_b(q.Kmin_b) )
+ * `ws` as for critiprefill_estimate (critiprefill_workspace_bytes of the same p is enough). */
+int critiprefill_decode_estimate(const cp_params* p, const void* q_last, const void* K, double* S_out, void* ws,
+                                 size_t ws_bytes, void* cuda_stream);
+
+/* Critical blocks of the last token from critiprefill_decode_estimate's scores:
+ *   idx  out  device, [B,Hq,k] int32 ascending, -1 padded: the last block (which holds the token) always, then the
+ *             k-1 other blocks with the largest score, ties to the larger index (forced_blocks and
+ *             CP_FLAG_SHARED_GROUP_LISTS apply as in critiprefill_select)
+ *   cnt  out  device, [B,Hq] int32 = min(k, n2) */
+int critiprefill_decode_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws,
+                               size_t ws_bytes, void* cuda_stream);
+
 /* Algorithm 2, lines 6-13, with token-level causality inside the listed blocks:
  *   O[t] = sum_{u in U_t} softmax_u(sm_scale * q_t.k_u) v_u,
  *   U_t  = { u <= t : floor(u/block_size) in idx[b,h,j,0:cnt] },  j = floor(t/segment_size).

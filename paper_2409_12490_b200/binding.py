@@ -27,6 +27,7 @@ EXPORTS = (
     "critiprefill_workspace_bytes", "critiprefill_estimate", "critiprefill_select",
     "critiprefill_attention", "critiprefill_dense_attention", "critiprefill_device_status",
     "critiprefill_estimate_static", "critiprefill_static_scratch_bytes",
+    "critiprefill_decode_estimate", "critiprefill_decode_select",
     "critiprefill_status_string",
 )
 
@@ -70,6 +71,8 @@ def load_library() -> ctypes.CDLL:
         lib.critiprefill_dense_attention.argtypes = [PP, P, P, P, P, P, P, SZ, P]
         lib.critiprefill_device_status.argtypes = [P, ctypes.POINTER(ctypes.c_int32), P]
         lib.critiprefill_estimate_static.argtypes = [PP, P, P, P, P, P]
+        lib.critiprefill_decode_estimate.argtypes = [PP, P, P, P, P, SZ, P]
+        lib.critiprefill_decode_select.argtypes = [PP, P, P, P, P, SZ, P]
         lib.critiprefill_static_scratch_bytes.argtypes = []
         lib.critiprefill_status_string.argtypes = [ctypes.c_int]
         lib.critiprefill_status_string.restype = ctypes.c_char_p
@@ -204,6 +207,27 @@ def select(prob: Problem, S, ws, idx=None, cnt=None):
     p = prob.params()
     _check(load_library().critiprefill_select(ctypes.byref(p), _ptr(S), _ptr(idx), _ptr(cnt), _ptr(ws), ws.numel(),
                                               _stream()), "critiprefill_select")
+    return idx, cnt
+
+
+def decode_estimate(prob: Problem, q_last, K, ws, S_out=None) -> torch.Tensor:
+    """critiprefill_decode_estimate: ln S [B,Hq,n2] fp64 of the last query token (Section 2.1)."""
+    assert q_last.is_contiguous() and q_last.shape == (prob.batch, prob.n_q_heads, prob.head_dim)
+    if S_out is None:
+        S_out = torch.empty((prob.batch, prob.n_q_heads, prob.n2), dtype=torch.float64, device=K.device)
+    p = prob.params(K=K)
+    _check(load_library().critiprefill_decode_estimate(ctypes.byref(p), _ptr(q_last), _ptr(K), _ptr(S_out), _ptr(ws),
+                                                       ws.numel(), _stream()), "critiprefill_decode_estimate")
+    return S_out
+
+
+def decode_select(prob: Problem, S, ws):
+    """critiprefill_decode_select: (idx [B,Hq,k] int32, cnt [B,Hq] int32) for the last query token."""
+    idx = torch.empty((prob.batch, prob.n_q_heads, prob.budget_blocks), dtype=torch.int32, device=S.device)
+    cnt = torch.empty((prob.batch, prob.n_q_heads), dtype=torch.int32, device=S.device)
+    p = prob.params()
+    _check(load_library().critiprefill_decode_select(ctypes.byref(p), _ptr(S), _ptr(idx), _ptr(cnt), _ptr(ws), ws.numel(),
+                                                     _stream()), "critiprefill_decode_select")
     return idx, cnt
 
 

@@ -88,6 +88,44 @@ int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32
   return launch_select(*p, m, S, idx, cnt, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int critiprefill_decode_estimate(const cp_params* p, const void* q_last, const void* K, double* S_out, void* ws,
+                                 size_t ws_bytes, void* cuda_stream) {
+  Dims m;
+  int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  if (!q_last || !K || !S_out) return CP_ERR_NULL;
+  if (!aligned16(q_last) || !aligned16(K)) return CP_ERR_SHAPE;
+  if (m.n2 > kMaxBlocksN2) return CP_ERR_UNSUPPORTED;
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  // Algorithm 1 on one segment that holds the last token alone: one "segment" per head that sees every block
+  Dims md = m;
+  md.n1 = 1; md.seg = m.n; md.r = 1;
+  cp_params pd = *p;
+  pd.flags &= ~CP_FLAG_MASK_BEFORE_SOFTMAX;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  char* w = static_cast<char*>(ws);
+  if ((rc = launch_summarize(pd, md, nullptr, K, w, s)) != CP_OK) return rc;
+  const WsLayout wl = ws_layout(md);
+  const size_t q_bytes = size_t(m.B) * m.Hq * m.d * m.es;      // Qmax = Qmin = q
+  if (cudaMemcpyAsync(w + wl.qmax, q_last, q_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(w + wl.qmin, q_last, q_bytes, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return CP_ERR_CUDA;
+  return launch_score(pd, md, w, nullptr, S_out, s);
+}
+
+int critiprefill_decode_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws, size_t ws_bytes,
+                               void* cuda_stream) {
+  Dims m;
+  int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  if (!S || !idx || !cnt) return CP_ERR_NULL;
+  if (m.n2 > kMaxBlocksN2) return CP_ERR_UNSUPPORTED;
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  Dims md = m;
+  md.n1 = 1; md.r = 1;                       // one row per head; its only "diagonal" block is the last block
+  return launch_select(*p, md, S, idx, cnt, static_cast<cudaStream_t>(cuda_stream), m.n2 - 1);
+}
+
 int critiprefill_attention(const cp_params* p, const void* Q, const void* K, const void* V, const int32_t* idx,
                            const int32_t* cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
   return attention_common(p, Q, K, V, idx, cnt, O, lse, ws, ws_bytes, cuda_stream, false);

@@ -70,7 +70,7 @@ int launch_lse(const cp_params& p, const Dims& m, char* ws, cudaStream_t s);   /
 int launch_score_generic(const cp_params& p, const Dims& m, const char* ws, const double* S_prev,
                          double* S_out, double* stats_out, cudaStream_t s);
 int launch_select(const cp_params& p, const Dims& m, const double* S, int32_t* idx, int32_t* cnt,
-                  cudaStream_t s);
+                  cudaStream_t s, int past_fixed = -1);
 int launch_attention_simt(const cp_params& p, const Dims& m, const void* Q, const void* K,
                           const void* V, const int32_t* idx, const int32_t* cnt, void* O, float* lse,
                           DeviceStatus* st, bool dense, cudaStream_t s);

@@ -49,7 +49,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int lane, int warp, i
 template <int KPT>
 __global__ void __launch_bounds__(kThreads)
 select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* __restrict__ cnt,
-              int n1, int n2, int r, int k, int pool, int n_sink, int n_local) {
+              int n1, int n2, int r, int k, int pool, int n_sink, int n_local, int past_fixed) {
   __shared__ unsigned int hist[256];
   __shared__ int warp_sum[kWarps];
   __shared__ unsigned long long prefix_sh;
@@ -61,7 +61,7 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
   const int unit = (blockIdx.x / n1) * pool * n1 + j;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const double* row = S + size_t(unit) * n2;
-  const int past = j * r;
+  const int past = past_fixed >= 0 ? past_fixed : j * r;   // past_fixed: the caller names the first diagonal block (decoding: the last block)
   const int rj = min(n2, past + r) - past;   // diagonal blocks of this segment (fewer in a short last segment)
   const int m = k - rj;
 
@@ -188,17 +188,17 @@ select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* 
 }  // namespace
 
 int launch_select(const cp_params& p, const Dims& m, const double* S, int32_t* idx, int32_t* cnt,
-                  cudaStream_t st) {
+                  cudaStream_t st, int past_fixed) {
   const int pool = (p.flags & CP_FLAG_SHARED_GROUP_LISTS) ? m.g : 1;
   const int n_sink = p.forced_blocks & 0xffff, n_local = (p.forced_blocks >> 16) & 0xffff;
   const long long units = (long long)m.B * (m.Hq / pool) * m.n1;
   if (units > 0x7fffffffLL) return CP_ERR_UNSUPPORTED;
   const int kpt = (m.n2 + kThreads - 1) / kThreads;
   const unsigned grid = unsigned(units);
-  if (kpt <= 4) select_kernel<4><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
-  else if (kpt <= 8) select_kernel<8><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
-  else if (kpt <= 16) select_kernel<16><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
-  else if (kpt <= 32) select_kernel<32><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local);
+  if (kpt <= 4) select_kernel<4><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local, past_fixed);
+  else if (kpt <= 8) select_kernel<8><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local, past_fixed);
+  else if (kpt <= 16) select_kernel<16><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local, past_fixed);
+  else if (kpt <= 32) select_kernel<32><<<grid, kThreads, 0, st>>>(S, idx, cnt, m.n1, m.n2, m.r, m.k, pool, n_sink, n_local, past_fixed);
   else return CP_ERR_UNSUPPORTED;
   return check_launch();
 }

@@ -223,6 +223,7 @@ int launch_summarize(const cp_params& p, const Dims& m, const void* Q, const voi
   };
   Side q = mk(Q, p.q_stride, m.Hq, m.seg, ws + w.qmax, ws + w.qmin);
   Side k = mk(K, p.k_stride, m.Hkv, m.blk, ws + w.kmax, ws + w.kmin);
+  if (Q == nullptr) q.n_groups = 0;          // key side only (the caller supplies the query representatives itself)
   k.oabs = reinterpret_cast<float*>(ws + w.kabs);
   const long long q_ctas = (q.n_groups + q.groups_per_cta - 1) / q.groups_per_cta;
   const long long k_ctas = (k.n_groups + k.groups_per_cta - 1) / k.groups_per_cta;

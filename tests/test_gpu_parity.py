@@ -202,6 +202,23 @@ def test_selection_variants_match_oracle(n_sink, n_local, shared):
     assert np.array_equal(it.cpu().numpy(), ir) and np.array_equal(ct.cpu().numpy(), cr)
 
 
+@pytest.mark.parametrize("name,blk", [("small_bf16", 64), ("small_bf16", 32), ("C1", 32)])
+def test_decode_phase_criticality_matches_oracle(name, blk):
+    """The last token's block criticality (Section 2.1) and its block list: bf16 (tensor-core log-sum-exp path) and fp32."""
+    cfg = CONFIGS.get(name, SMALL_BF16).with_(block_size=blk)
+    Q, K, _ = make_qkv(cfg)
+    prob = problem(cfg)
+    ws = cp.alloc_workspace(prob)
+    q_last = Q[:, :, -1].contiguous()
+    S = cp.decode_estimate(prob, q_last.cuda(), K.cuda(), ws)
+    idx, cnt = cp.decode_select(prob, S, ws)
+    assert cp.device_status(ws) == 0
+    S_ref = oracle.decode_estimate(q_last, K, cfg.block_size, est_scale=f32(cfg.est_scale))
+    assert np.abs(S.cpu().numpy() - S_ref).max() <= 1e-9
+    idx_ref, cnt_ref = oracle.decode_select(S_ref, cfg.budget_blocks)
+    assert np.array_equal(idx.cpu().numpy(), idx_ref) and np.array_equal(cnt.cpu().numpy(), cnt_ref)
+
+
 def test_bad_list_sets_bounds_status_without_faulting():
     cfg = SMALL_BF16
     Q, K, V = make_qkv(cfg)
