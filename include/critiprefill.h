@@ -169,10 +169,14 @@ int critiprefill_decode_select(const cp_params* p, const double* S, int32_t* idx
  *   O[t] = sum_{u in U_t} softmax_u(sm_scale * q_t.k_u) v_u,
  *   U_t  = { u <= t : floor(u/block_size) in idx[b,h,j,0:cnt] },  j = floor(t/segment_size).
  *   Q, K, V   in   device
- *   idx, cnt  in   device, as produced by critiprefill_select.  Contract per list: ascending,
- *                  unique, r_j <= cnt <= k, and its last r_j entries are exactly the diagonal
- *                  blocks j*r .. min(n2,(j+1)*r)-1.  A list that breaks it sets CP_ERR_BOUNDS in the
- *                  status block and its segment's rows of O are not written.
+ *   idx, cnt  in   device.  Contract per list (Algorithm 2 takes any index set I): 0 <= cnt <= k
+ *                  entries, ascending, unique, each a block segment j can see, 0 <= b < min(n2, (j+1)*r).
+ *                  Lists of the form critiprefill_select emits (past blocks, then exactly the diagonal
+ *                  blocks) take the fast tile sequence; any other valid list is served element by
+ *                  element masking (a listed diagonal block gets the causal mask wherever it sits).
+ *                  A row that sees no key at all (possible only when diagonal blocks are left out)
+ *                  gets O = 0 and lse = -inf.  A list that breaks the contract sets CP_ERR_BOUNDS in
+ *                  the status block and its segment's rows of O are not written.
  *   O         out  device, same dtype and layout family as Q (o_stride)
  *   lse       out  device, nullable, [B,Hq,n] fp32: ln sum_{u in U_t} exp(sm_scale*q_t.k_u)
  * bf16 / fp16: operands in that type, fp32 accumulation, probabilities rounded to that type

@@ -19,15 +19,14 @@ template <> __device__ __forceinline__ __half from_f32<__half>(float x) { return
 template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
-// The list contract: ascending, in range, last r entries are the diagonal blocks of segment j.
+// The list contract: at most k entries, ascending, unique, each a block that segment j can see.
 __device__ __forceinline__ bool list_ok(const int32_t* list, int c, int j, int r_full, int n2, int k, int lane) {
-  const int r = min(n2, (j + 1) * r_full) - j * r_full;   // diagonal blocks of segment j
-  bool ok = (c >= r) && (c <= k);
+  const int vis = min(n2, (j + 1) * r_full);
+  bool ok = (c >= 0) && (c <= k);
   if (ok) {
     for (int i = lane; i < c; i += 32) {
       const int v = list[i];
-      if (i >= c - r) ok = ok && (v == j * r_full + (i - (c - r)));
-      else ok = ok && (v >= 0) && (v < j * r_full) && (i == 0 || list[i - 1] < v);
+      ok = ok && (v >= 0) && (v < vis) && (i == 0 || list[i - 1] < v);
     }
   }
   return __all_sync(0xffffffffu, ok);
@@ -111,7 +110,7 @@ attention_simt_kernel(const T* __restrict__ Q, const T* __restrict__ K, const T*
     }
   }
   T* o = O + b * osb + h * osh + int64_t(t) * ost;
-  const float inv = 1.f / l_run;
+  const float inv = l_run > 0.f ? 1.f / l_run : 0.f;   // a row without any visible key: zeros, lse = ln 0
 #pragma unroll
   for (int i = 0; i < CPL; ++i) o[lane + 32 * i] = from_f32<T>(acc[i] * inv);
   if (lse != nullptr && lane == 0) lse[rowid] = m_run + logf(l_run);

@@ -55,6 +55,9 @@ struct Unit {
   int seg_j;
   int rj;           // diagonal blocks of the segment (r, fewer in a short last segment)
   int cnt;
+  int generic;      // the list is not "past blocks, then exactly the diagonal blocks": every listed block is gathered and
+                    // every tile is masked element by element (a key counts iff its token is not after the query's)
+  int rowsB;        // the unit has a second 128-row query tile
 };
 
 struct Bars {
@@ -107,7 +110,8 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
 // Units are ordered KV-head-major so that CTAs resident at the same time share K/V tiles in
 // L2; within a KV head the dense kernel takes the longest rows first.
 // `cnt` is the unit's list length when the caller already has it, kLoadCnt to read it from global memory.
-constexpr int kLoadCnt = -2, kBadList = -1, kEmptyUnit = -3;   // kEmptyUnit: no query row of the unit lies inside the sequence
+constexpr int kLoadCnt = -2, kBadList = -1, kEmptyUnit = -3, kZeroUnit = -4;   // kEmptyUnit: no query row of the unit lies inside the sequence;
+                                                                                // kZeroUnit: an empty list -- the unit's rows are zeros
 __device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
   Unit u;
   u.list = nullptr;
@@ -149,25 +153,35 @@ __device__ __forceinline__ Unit decode_unit(const Args& a, int x, int cnt) {
     u.c_tok = j * a.seg; u.n_cont = 2 * p; u.d_tok = u.q_tok;
     u.nB = (2 * p + 1 < q_tiles && u.q_tok + kTile < a.n) ? 1 : 0;   // tile B exists and starts inside the sequence
   }
+  u.generic = 0;
+  u.rowsB = u.nB ? 1 : 0;
   u.nA = u.n_past_tiles + u.n_cont + 1;       // up to and including its own diagonal tile
   u.nB = u.nB ? u.nA + 1 : 0;                 // one more diagonal tile; 0 when the segment has an odd tile count
   u.T = u.nB ? u.nB : u.nA;
   return u;
 }
 
-// The list contract, checked by the producer warp before it publishes a unit: r <= cnt <= k,
-// ascending past blocks, then exactly the r diagonal blocks of the segment.
-__device__ __forceinline__ bool unit_ok(const Args& a, const Unit& u, int lane) {
-  if (a.dense) return true;
-  bool ok = (u.cnt >= u.rj) && (u.cnt <= a.k);
-  if (ok) {
+// The list contract, checked by the producer warp before it publishes a unit: at most k entries, ascending, unique,
+// each a block the segment can see (0 <= b < (j+1)*r).  Returns 0 when the list has the form the selection emits
+// (past blocks, then exactly the diagonal blocks of the segment: the fast tile sequence applies), 1 for any other
+// valid list (generic tile sequence), -1 for a list that breaks the contract.
+__device__ __forceinline__ int classify_unit(const Args& a, const Unit& u, int lane) {
+  if (a.dense) return 0;
+  const int vis = min(a.n2, (u.seg_j + 1) * a.r);
+  bool gen_ok = (u.cnt >= 0) && (u.cnt <= a.k);
+  bool std_ok = gen_ok && (u.cnt >= u.rj);
+  if (gen_ok) {
     for (int i = lane; i < u.cnt; i += 32) {
       const int v = u.list[i];
-      if (i >= u.n_past) ok = ok && (v == u.seg_j * a.r + (i - u.n_past));
-      else ok = ok && v >= 0 && v < u.seg_j * a.r && (i == 0 || u.list[i - 1] < v);
+      const bool asc = v >= 0 && v < vis && (i == 0 || u.list[i - 1] < v);
+      gen_ok = gen_ok && asc;
+      if (i >= u.n_past) std_ok = std_ok && (v == u.seg_j * a.r + (i - u.n_past));
+      else std_ok = std_ok && asc && v < u.seg_j * a.r;
     }
   }
-  return __all_sync(0xffffffffu, ok);
+  gen_ok = __all_sync(0xffffffffu, gen_ok);
+  std_ok = __all_sync(0xffffffffu, std_ok);
+  return !gen_ok ? -1 : (std_ok ? 0 : 1);
 }
 
 __device__ __forceinline__ bool stop_requested(const Args& a, Bars* bars) {
@@ -192,9 +206,23 @@ __device__ __forceinline__ bool publish_unit(const Args& a, Bars* bars, uint32_t
     cnt = u_out->cnt;
     if (u_out->q_tok >= a.n) {
       cnt = kEmptyUnit;                               // a short last segment has fewer units
-    } else if (!unit_ok(a, *u_out, lane)) {
-      if (lane == 0) report(a.st, CP_ERR_BOUNDS, 1, u_out->b, u_out->h, u_out->seg_j, u_out->cnt);
-      cnt = kBadList;
+    } else {
+      const int cls = classify_unit(a, *u_out, lane);
+      if (cls < 0) {
+        if (lane == 0) report(a.st, CP_ERR_BOUNDS, 1, u_out->b, u_out->h, u_out->seg_j, u_out->cnt);
+        cnt = kBadList;
+      } else if (cls == 1) {
+        // any other valid list: all listed blocks are gathered, both query tiles consume every tile
+        u_out->generic = 1;
+        u_out->n_past = cnt;
+        u_out->n_past_tiles = (cnt * a.blk + kTile - 1) / kTile;
+        u_out->last_cols = cnt * a.blk - (u_out->n_past_tiles - 1) * kTile;
+        u_out->n_cont = 0;
+        u_out->nA = u_out->n_past_tiles;
+        u_out->nB = u_out->rowsB ? u_out->n_past_tiles : 0;
+        u_out->T = u_out->n_past_tiles;
+        if (u_out->T == 0) cnt = kZeroUnit;           // nothing listed: the rows are zeros
+      }
     }
   }
   u_out->cnt = cnt;
@@ -218,7 +246,7 @@ __device__ __forceinline__ bool receive_unit(const Args& a, Bars* bars, uint32_t
 }
 
 // ---------------------------------------------------------------- softmax role
-constexpr int kMaskNone = 0, kMaskCausal = 1, kMaskCols = 2;
+constexpr int kMaskNone = 0, kMaskCausal = 1, kMaskCols = 2, kMaskGeneric = 3;
 
 template <bool kF16>
 __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int which, int warp_in_wg, int lane) {
@@ -236,6 +264,17 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     Unit u;
     if (!receive_unit(a, bars, q, lane, &x, &u) || x >= a.n_units || bars->abort_flag) return;
     if (u.cnt == kBadList || u.cnt == kEmptyUnit) continue;
+    if (u.cnt == kZeroUnit) {
+      // an empty list: no key is visible to any row of the unit -- zeros, and lse = ln 0
+      const int t = u.q_tok + which * kTile + row;
+      if ((which == 0 || u.rowsB) && t < a.n) {
+        uint4* dst = reinterpret_cast<uint4*>(a.O + u.b * a.osb + u.h * a.osh + int64_t(t) * a.ost);
+#pragma unroll
+        for (int i = 0; i < kD * 2 / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (a.lse != nullptr) a.lse[((long long)u.b * a.Hq + u.h) * a.n + t] = -CUDART_INF;
+      }
+      continue;
+    }
     const int my_tiles = which == 0 ? u.nA : u.nB;
     if (my_tiles == 0) continue;                        // this unit has no tile B
     float m_run = -CUDART_INF, l_run = 0.f;
@@ -253,9 +292,32 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
       float* s = reinterpret_cast<float*>(sv);
 
       int kind = kMaskNone, cols = kTile;
-      if (jt == my_tiles - 1) kind = kMaskCausal;                                   // own diagonal tile
+      if (u.generic) kind = kMaskGeneric;
+      else if (jt == my_tiles - 1) kind = kMaskCausal;                              // own diagonal tile
       else if (jt == u.n_past_tiles - 1 && u.last_cols < kTile) { kind = kMaskCols; cols = u.last_cols; }
-      if (kind == kMaskCausal) {
+      if (kind == kMaskGeneric) {
+        // a gathered tile of a generic list: the tile holds 128/blk listed blocks; key column i belongs to token
+        // list[...]*blk + i % blk and counts iff that token is not after this row's token.  lim[q] = last visible
+        // offset inside sub-block q (-1: none, also for sub-blocks beyond the list)
+        const int t_row = u.q_tok + which * kTile + row;
+        const int bpt = kTile / a.blk;
+        int lim[4];
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) {
+          const int li = jt * bpt + qq;
+          lim[qq] = (qq < bpt && li < u.cnt) ? t_row - __ldg(u.list + li) * a.blk : -1;
+        }
+        if (a.blk == 128) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) s[i] = (i > lim[0]) ? -CUDART_INF : s[i];
+        } else if (a.blk == 64) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) s[i] = ((i & 63) > lim[i >> 6]) ? -CUDART_INF : s[i];
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) s[i] = ((i & 31) > lim[i >> 5]) ? -CUDART_INF : s[i];
+        }
+      } else if (kind == kMaskCausal) {
 #pragma unroll
         for (int i = 0; i < 128; ++i) s[i] = (i > row) ? -CUDART_INF : s[i];
       } else if (kind == kMaskCols) {
@@ -289,7 +351,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
         }
       }
       CP_STAMP(tr, which * 1024 + jt * 8 + 3);
-      const float neg_mc = -m_run * c;
+      const float neg_mc = (m_run == -CUDART_INF) ? 0.f : -m_run * c;   // a row that has not seen a key yet (generic lists only): exp2(-inf) = 0
       const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
       float2 sum2 = make_float2(0.f, 0.f);
       uint32_t pk[64];
@@ -330,7 +392,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     tc_fence_after();
     const int t = u.q_tok + which * kTile + row;
     uint16_t* orow = a.O + u.b * a.osb + u.h * a.osh + int64_t(t) * a.ost;
-    const float inv = 1.f / l_run;
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;   // a row without any visible key (generic lists only): zeros
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       uint32_t ov[32];
@@ -376,7 +438,7 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
     if (stop_requested(a, bars)) { bars->abort_flag = 1; return; }
     const Unit u_cur = u;
     if (!publish_unit(a, bars, q + 1, lane, &x, &u)) return;
-    if (u_cur.cnt == kBadList || u_cur.cnt == kEmptyUnit) continue;
+    if (u_cur.cnt == kBadList || u_cur.cnt == kEmptyUnit || u_cur.cnt == kZeroUnit) continue;
     // Q tiles: the buffer is free once every QK^T of the previous unit has completed
     if (n_units > 0 && !mbar_wait(&bars->q_empty, (n_units - 1) & 1, bars, a.st, 31)) return;
     if (lane == 0) {
@@ -452,7 +514,7 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
     int x;
     Unit u;
     if (!receive_unit(a, bars, q, lane, &x, &u) || x >= a.n_units || bars->abort_flag) return;
-    if (u.cnt == kBadList || u.cnt == kEmptyUnit) continue;
+    if (u.cnt == kBadList || u.cnt == kEmptyUnit || u.cnt == kZeroUnit) continue;
     const int T = u.T, TA = u.nA;
     const bool hasB = u.nB > 0;
     if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;

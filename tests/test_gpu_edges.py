@@ -288,3 +288,61 @@ def test_layer_replays_from_a_cuda_graph():
     assert cp.device_status(ws) == 0
     assert torch.equal(O, O1_eager) and torch.equal(idx, idx1_eager)
     assert not torch.equal(O1_eager, O_eager)
+
+
+@pytest.mark.parametrize("flags", [0, cp.FLAG_FORCE_SIMT])
+@pytest.mark.parametrize("blk,k", [(32, 14), (64, 9), (128, 6)])
+def test_any_ascending_list_of_visible_blocks_is_accepted(blk, k, flags):
+    """Algorithm 2 takes any index set: lists with diagonal blocks missing, out of their usual place or alone, empty
+    lists (rows of zeros, lse = -inf), and lists of the usual form, mixed over the segments of one call."""
+    cfg = BASE.with_(seq_len=2048, n_q_heads=4, n_kv_heads=2, segment_size=256, block_size=blk, budget_tokens=k * blk)
+    Q, K, V = make_qkv(cfg)
+    r, n1 = cfg.r, cfg.n1
+    rng = np.random.default_rng(blk + k)
+    idx = np.full((1, 4, n1, k), -1, dtype=np.int32)
+    cnt = np.zeros((1, 4, n1), dtype=np.int32)
+    for h in range(4):
+        for j in range(n1):
+            vis = (j + 1) * r
+            mode = (h + j) % 5
+            if mode == 0:
+                sel = []                                                     # nothing listed
+            elif mode == 1:
+                sel = sorted(rng.choice(vis, size=min(k, vis, 1 + int(rng.integers(k))), replace=False).tolist())   # any visible blocks
+            elif mode == 2:
+                sel = [j * r + int(rng.integers(r))]                         # a single diagonal block
+            elif mode == 3:
+                past = sorted(rng.choice(max(j * r, 1), size=min(max(k - r, 0), j * r), replace=False).tolist()) if j else []
+                sel = past + list(range(j * r, (j + 1) * r))                 # the usual form
+                sel = sel[-k:] if len(sel) > k else sel
+                sel = sorted(set(sel))
+            else:
+                sel = sorted(set(range(j * r, (j + 1) * r, 2)) | ({0} if j else set()))[:k]   # every other diagonal block
+            cnt[0, h, j] = len(sel)
+            idx[0, h, j, :len(sel)] = sel
+    prob = problem(cfg, flags=flags)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = to_dev(Q, K, V)
+    O, lse = cp.attention(prob, Qd, Kd, Vd, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), ws, want_lse=True)
+    assert cp.device_status(ws) == 0
+    O_ref, lse_ref = oracle.sparse_attention(Q, K, V, idx, cnt, cfg.segment_size, cfg.block_size, f32(1.0 / np.sqrt(cfg.head_dim)))
+    assert_attention_close(O, O_ref)
+    lse_gpu = lse.cpu().numpy()
+    none = np.isneginf(lse_ref)
+    assert none.any() and np.array_equal(np.isneginf(lse_gpu), none)         # rows without any visible key
+    assert (O.float().cpu().numpy()[none] == 0).all()
+    assert np.abs(lse_gpu[~none] - lse_ref[~none]).max() <= 2e-3
+    # a list that is not ascending, or reaches a block the segment cannot see, still sets CP_ERR_BOUNDS
+    for bad_val, pos in ((10 ** 6, 0), (None, 1)):
+        bad = idx.copy()
+        jb = n1 - 1
+        full = np.arange(k, dtype=np.int32)
+        bad[0, 1, jb] = full
+        bad_cnt = cnt.copy(); bad_cnt[0, 1, jb] = k
+        if bad_val is None:
+            bad[0, 1, jb, 1] = bad[0, 1, jb, 0]                                  # duplicate entry
+        else:
+            bad[0, 1, jb, k - 1] = bad_val
+        ws.zero_()
+        cp.attention(prob, Qd, Kd, Vd, torch.from_numpy(bad).cuda(), torch.from_numpy(bad_cnt).cuda(), ws)
+        assert cp.device_status(ws) == 7
