@@ -137,3 +137,25 @@ def test_C4_scores_selection_all_heads_and_dense_rows_per_head():
     rows = np.array(rows, dtype=np.int64)
     Od_ref, _ = oracle.dense_attention_rows(Q, K, V, f32(1.0 / np.sqrt(cfg.head_dim)), rows)
     assert_attention_close(Od[rows[:, 0], rows[:, 1], rows[:, 2]], Od_ref, label=f"C4 dense, 64 rows of each of {cfg.n_q_heads} heads")
+
+
+def test_mass_recall_from_the_kernels_lse_equals_the_oracles():
+    """The accuracy diagnostic the benchmark reports -- the share of a row's dense softmax mass that the listed keys
+    hold, exp(lse_sparse - lse_dense) from the two kernels -- against the same quantity from the oracle, on C3."""
+    cfg = CONFIGS["C3"].with_(name="C3 recall", budget_tokens=1024)
+    Q, K, V = make_qkv(cfg)
+    prob, ws, (Qd, Kd, Vd), O, S, idx, cnt = _run_layer(cfg, Q, K, V)
+    _, lse_s = cp.attention(prob, Qd, Kd, Vd, idx, cnt, ws, want_lse=True)
+    _, lse_d = cp.dense_attention(prob, Qd, Kd, Vd, ws, want_lse=True)
+    assert cp.device_status(ws) == 0
+    rows = _unit_rows(cfg, 32, 16, seed=5)
+    sm = f32(1.0 / np.sqrt(cfg.head_dim))
+    _, ls_ref = oracle.sparse_attention_rows(Q, K, V, idx.cpu().numpy(), cnt.cpu().numpy(), cfg.segment_size, cfg.block_size, sm, rows)
+    _, ld_ref = oracle.dense_attention_rows(Q, K, V, sm, rows)
+    recall_ref = np.exp(ls_ref - ld_ref)
+    sel = (rows[:, 0], rows[:, 1], rows[:, 2])
+    recall_gpu = torch.exp(lse_s.double() - lse_d.double())[sel].cpu().numpy()
+    assert ((recall_ref > 0) & (recall_ref <= 1 + 1e-12)).all()
+    assert np.abs(recall_gpu - recall_ref).max() <= 5e-3, np.abs(recall_gpu - recall_ref).max()
+    print(f"[parity] mass recall on {len(rows)} rows: max abs diff {np.abs(recall_gpu - recall_ref).max():.2e}, "
+          f"median recall {np.median(recall_ref):.3f}")
