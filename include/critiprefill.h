@@ -64,6 +64,9 @@ enum {
   CP_FLAG_TEST_WITHHOLD_V = 4,     /* test hook for the bounded waits of the tensor-core kernel: V tiles are
                                       never loaded, so a pipeline wait expires after about 2 s, the kernel
                                       drains and the status block reads CP_ERR_TIMEOUT (outputs invalid) */
+  CP_FLAG_FORCE_SPLIT_SCORE = 16,  /* estimate: take the two-kernel score path (tensor-core log-sum-exps + exact logits of
+                                      the visible blocks) whatever the size of the score map; without the flag it is used
+                                      from a few million scores up, where it is faster (16-bit inputs, head_dim 128) */
   CP_FLAG_SHARED_GROUP_LISTS = 8   /* select: one list per KV group instead of one per query head -- the g query
                                       heads of a KV head all receive the list selected from the element-wise
                                       maximum of their scores (a variant; the paper describes a single head) */

@@ -22,6 +22,7 @@ FLAG_MASK_BEFORE_SOFTMAX = 1
 FLAG_FORCE_SIMT = 2
 FLAG_TEST_WITHHOLD_V = 4
 FLAG_SHARED_GROUP_LISTS = 8
+FLAG_FORCE_SPLIT_SCORE = 16
 
 EXPORTS = (
     "critiprefill_workspace_bytes", "critiprefill_estimate", "critiprefill_select",

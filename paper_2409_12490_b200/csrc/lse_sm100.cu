@@ -109,7 +109,10 @@ lse_sm100_kernel(const __grid_constant__ CUtensorMap tmKmax, const __grid_consta
   const int h0 = (kvh % Hkv) * a.g + sub * a.U;
   const int j0 = qchunk * a.segs_per_cta;
   // row m of the CTA: column group m/8 = (4-segment chunk c4, head u); within it (segment s, representative)
-  auto row_seg = [&](int m) { return j0 + ((m >> 3) / a.U) * 4 + ((m >> 1) & 3); };
+  auto row_seg = [&](int m) {            // rows beyond the CTA's share of segments (or beyond n1) map past the end: unused
+    const int local = ((m >> 3) / a.U) * 4 + ((m >> 1) & 3);
+    return local < a.segs_per_cta ? j0 + local : a.n1;
+  };
   auto row_unit = [&](int m) { return (size_t(b) * a.Hq + h0 + (m >> 3) % a.U) * a.n1 + row_seg(m); };
   auto row_limit = [&](int m) {          // blocks [0, limit) enter the row's softmax
     const int j = row_seg(m);
@@ -206,6 +209,9 @@ lse_sm100_kernel(const __grid_constant__ CUtensorMap tmKmax, const __grid_consta
     const uint32_t t_row = tm + (uint32_t((warp & 3) * 32) << 16);
     const float es = a.es, l2e = 1.4426950408889634f;
     float flagT = -CUDART_INF_F, mref_l2 = 0.f;
+#ifdef CP_LSE_DEBUG
+    long long dbg_wait = 0, dbg_a = 0, dbg_b = 0;
+#endif
     const float es_l2 = es * l2e;
     for (uint32_t it = uint32_t(my_kr); it < n_items; it += 2) {
       const uint32_t stage = it % kStages;
@@ -219,7 +225,14 @@ lse_sm100_kernel(const __grid_constant__ CUtensorMap tmKmax, const __grid_consta
         flagT = (eps < 4.f) ? Mx - window : -CUDART_INF_F;     // eps too large (or NaN): flag everything
         mref_l2 = Mx * l2e;
       }
+#ifdef CP_LSE_DEBUG
+      const long long tw0 = clock64();
+#endif
       if (!mbar_wait(&bars->acc_full[stage], (it / kStages) & 1, &bars->abort_flag, a.st, 63)) break;
+#ifdef CP_LSE_DEBUG
+      const long long tw1 = clock64();
+      dbg_wait += tw1 - tw0;
+#endif
       tc_fence_after();
       const uint32_t t_acc = t_row + stage * kTileN;
       uint32_t va[32], vb[32];
@@ -269,7 +282,16 @@ lse_sm100_kernel(const __grid_constant__ CUtensorMap tmKmax, const __grid_consta
       tmem_wait_ld(); piece_fn(vb, 3);
       tc_fence_before();
       mbar_arrive(&bars->acc_empty[stage]);
+#ifdef CP_LSE_DEBUG
+      if (sweep_b) dbg_b += clock64() - tw1; else dbg_a += clock64() - tw1;
+#endif
     }
+#ifdef CP_LSE_DEBUG
+    if (blockIdx.x == 0 && tid == 0) {
+      long long* dbg = reinterpret_cast<long long*>(reinterpret_cast<char*>(a.st) + 216);
+      dbg[0] = dbg_wait; dbg[1] = dbg_a; dbg[2] = dbg_b;
+    }
+#endif
   }
   tc_fence_before();
   __syncthreads();
@@ -462,7 +484,11 @@ int launch_lse(const cp_params& p, const Dims& m, char* ws, cudaStream_t st) {
   a.st = reinterpret_cast<DeviceStatus*>(ws);
   a.Hq = m.Hq; a.g = m.g; a.U = m.g % 4 == 0 ? 4 : (m.g % 2 == 0 ? 2 : 1);
   a.n1 = m.n1; a.n2 = m.n2; a.seg = m.seg; a.blk = m.blk;
+  // a CTA has 128 logit rows = 64 / U segments; on mid-sized problems fewer segments per CTA (rows left unused) put more
+  // SMs to work on the sweeps and the exact pass, which run per CTA one after the other
   a.segs_per_cta = 64 / a.U;
+  const long long per_chunk = (long long)m.B * m.Hkv * (m.g / a.U);
+  while (a.segs_per_cta > 4 && per_chunk * ((m.n1 + a.segs_per_cta - 1) / a.segs_per_cta) < 100) a.segs_per_cta /= 2;
   a.n_qchunks = (m.n1 + a.segs_per_cta - 1) / a.segs_per_cta;
   a.mask_first = (p.flags & CP_FLAG_MASK_BEFORE_SOFTMAX) ? 1 : 0;
   a.box_rows = m.n2 < kTileN ? m.n2 : kTileN;

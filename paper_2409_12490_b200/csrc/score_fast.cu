@@ -12,6 +12,10 @@ namespace {
 
 constexpr int kThreads = 384;   // 12 warps x <= 168 registers: one CTA per SM
 constexpr int kWarps = kThreads / 32;
+#ifndef CP_SCORE_FAST_MIN
+#define CP_SCORE_FAST_MIN 3000000
+#endif
+constexpr long long kFastMinScores = CP_SCORE_FAST_MIN;   // (batch x heads x segments x blocks) from which the two-kernel path is used
 constexpr int kG = 4;                       // segments per CTA: one MMA column group = 4 segments x {Qmax, Qmin} of one head
 
 // One CTA: G = 4 consecutive segments x U query heads of one KV group.  The fp64 MMA m16n8k16 runs with 16 key
@@ -189,7 +193,11 @@ int launch_visible_t(const Dims& m, const char* ws, const WsLayout& w, const dou
 // K2 dispatcher.  16-bit inputs with head_dim 128 take the two-kernel path (log-sum-exps, then exact logits of
 // the visible blocks); everything else the general kernel.
 int launch_score(const cp_params& p, const Dims& m, char* ws, const double* S_prev, double* S_out, cudaStream_t st) {
-  const bool fast = (p.dtype == CP_BF16 || p.dtype == CP_F16) && m.d == 128;
+  // The two-kernel path pays for an extra launch and for the serial sweeps of the log-sum-exp kernel; it wins once the
+  // score map is large (measured: 2x at 33 M scores, nothing below a few million), so small maps keep the general kernel.
+  const long long scores = (long long)m.B * m.Hq * m.n1 * m.n2;
+  const bool fast = (p.dtype == CP_BF16 || p.dtype == CP_F16) && m.d == 128 &&
+                    (scores >= kFastMinScores || (p.flags & CP_FLAG_FORCE_SPLIT_SCORE));
   if (!fast) return launch_score_generic(p, m, ws, S_prev, S_out, nullptr, st);
   const WsLayout w = ws_layout(m);
   int rc = launch_lse(p, m, ws, st);

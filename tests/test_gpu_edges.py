@@ -346,3 +346,41 @@ def test_any_ascending_list_of_visible_blocks_is_accepted(blk, k, flags):
         ws.zero_()
         cp.attention(prob, Qd, Kd, Vd, torch.from_numpy(bad).cuda(), torch.from_numpy(bad_cnt).cuda(), ws)
         assert cp.device_status(ws) == 7
+
+
+@pytest.mark.parametrize("case", ["gqa2_fused", "mha_batch3", "ragged", "mask_first", "fp16_scaled", "blk32_wide"])
+def test_split_score_path_on_small_ragged_and_variant_shapes(case):
+    """The two-kernel score path (tensor-core log-sum-exps + exact visible logits) is chosen by size; forced here on small
+    shapes so that its corner cases run against the oracle: 1, 2 and 4 heads per CTA, batch > 1, lengths that are not
+    multiples of the segment / block / tile sizes, the mask-first variant, fp16 with a logit scale, layer fusion."""
+    f = cp.FLAG_FORCE_SPLIT_SCORE
+    if case == "gqa2_fused":
+        cfg, flags = BASE.with_(seq_len=2048, n_q_heads=4, n_kv_heads=2, block_size=64, budget_tokens=512), f
+    elif case == "mha_batch3":
+        cfg, flags = BASE.with_(batch=3, n_q_heads=3, n_kv_heads=3, seq_len=1536, block_size=32, budget_tokens=384), f
+    elif case == "ragged":
+        cfg, flags = BASE.with_(seq_len=1340, n_q_heads=8, n_kv_heads=2, block_size=32, budget_tokens=320), f
+    elif case == "mask_first":
+        cfg, flags = BASE.with_(seq_len=2304, n_q_heads=4, n_kv_heads=1, block_size=64, budget_tokens=512), f | cp.FLAG_MASK_BEFORE_SOFTMAX
+    elif case == "fp16_scaled":
+        cfg, flags = BASE.with_(seq_len=2048, n_q_heads=4, n_kv_heads=2, dtype="f16", est_scale=f32(1.0 / np.sqrt(128.0))), f
+    else:
+        cfg, flags = BASE.with_(seq_len=9000, n_q_heads=4, n_kv_heads=1, segment_size=128, block_size=32, budget_tokens=512), f
+    Q, K, _ = make_qkv(cfg)
+    prob = problem(cfg, flags=flags)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd = to_dev(Q, K)
+    mf = bool(flags & cp.FLAG_MASK_BEFORE_SOFTMAX)
+    S0 = cp.estimate(prob, Qd, Kd, ws)
+    S0_ref = oracle_scores(cfg, Q, K, mask_before_softmax=mf)
+    compare_scores(S0, S0_ref)
+    # the general kernel must agree to the last bits it can (same representatives, fp64 on both sides)
+    S0_gen = cp.estimate(problem(cfg, flags=flags & ~f), Qd, Kd, ws)
+    fin = torch.isfinite(S0_gen)
+    assert torch.equal(torch.isneginf(S0), torch.isneginf(S0_gen)) and (S0[fin] - S0_gen[fin]).abs().max().item() <= 1e-10
+    # second layer fused onto the first
+    Q1, K1, _ = make_qkv(cfg, layer=1)
+    S1 = cp.estimate(prob, *to_dev(Q1, K1), ws, S_prev=S0)
+    compare_scores(S1, oracle_scores(cfg, Q1, K1, S_prev=S0_ref, mask_before_softmax=mf))
+    idx, cnt = cp.select(prob, S1, ws)
+    assert cp.device_status(ws) == 0
