@@ -610,6 +610,55 @@ def run_overlap(args, cfg):
     print(json.dumps({"token_critical_set_overlap": rows, "k": k, "tokens": n, "config": workload_config(cfg), "data": "synthetic"}))
 
 
+def run_projection(args, cfg):
+    """Upstream fusion (Eq. 1): the query / key projection kernel whose epilogue leaves the representatives of
+    Algorithm 1 in the workspace, timed beside the estimate with and without its own pass over Q and K.
+    Seeded random X and weights of the Llama3-8B width (d_model 4096); a kernel measurement, not the bench line."""
+    from paper_2409_12490_b200 import binding as cp
+    from paper_2409_12490_b200.build import build
+    build()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    d_model = args.d_model
+    g = torch.Generator(device=dev).manual_seed(20240912)
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[cfg.dtype]
+    X = torch.randn((cfg.batch, cfg.seq_len, d_model), generator=g, device=dev, dtype=torch.float32).to(tdt)
+    Wq = (torch.randn((cfg.n_q_heads * cfg.head_dim, d_model), generator=g, device=dev) / math.sqrt(d_model)).to(tdt)
+    Wk = (torch.randn((cfg.n_kv_heads * cfg.head_dim, d_model), generator=g, device=dev) / math.sqrt(d_model)).to(tdt)
+    inv = 500000.0 ** (-torch.arange(0, cfg.head_dim, 2, device=dev, dtype=torch.float64) / cfg.head_dim)
+    ang = torch.arange(cfg.seq_len, device=dev, dtype=torch.float64)[:, None] * inv[None, :]
+    cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    prob = cp.Problem.from_config(cfg)
+    ready = cp.Problem.from_config(cfg, flags=cp.FLAG_SUMMARIES_READY)
+    ws = cp.alloc_workspace(prob, dev)
+    Q, K = cp.project_qk(prob, X, Wq, Wk, ws, rope_cos=cos, rope_sin=sin)
+    S = cp.estimate(ready, Q, K, ws)
+    S2 = cp.estimate(prob, Q, K, ws)
+    same = bool(torch.equal(S, S2))
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    reps = max(3, min(args.steps, 10))
+    ev[0].record()
+    for _ in range(reps):
+        cp.project_qk(prob, X, Wq, Wk, ws, rope_cos=cos, rope_sin=sin, Q_out=Q, K_out=K)
+    ev[1].record()
+    for _ in range(reps):
+        cp.estimate(ready, Q, K, ws, S_out=S)
+    ev[2].record()
+    for _ in range(reps):
+        cp.estimate(prob, Q, K, ws, S_out=S)
+    ev[3].record()
+    torch.cuda.synchronize()
+    assert cp.device_status(ws) == 0
+    proj_ms, est_ready_ms, est_plain_ms = (ev[i].elapsed_time(ev[i + 1]) / reps for i in range(3))
+    flops = 2.0 * cfg.batch * cfg.seq_len * d_model * (cfg.n_q_heads + cfg.n_kv_heads) * cfg.head_dim
+    peaks = load_peaks()
+    print(json.dumps({"projection_ms": proj_ms, "gemm_tflops": flops / (proj_ms * 1e-3) / 1e12,
+                      "frac_of_bf16_peak": flops / (proj_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                      "estimate_ms_summaries_ready": est_ready_ms, "estimate_ms_with_own_pass": est_plain_ms,
+                      "scores_identical": same, "d_model": d_model, "config": workload_config(cfg), "data": "synthetic"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -626,6 +675,9 @@ def main():
                     help="token-wise critical-set overlap between neighbouring queries (Eq. 3; quality diagnostic) instead of the bench line")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
                     help="with --gpus N > 1: N independent layers (weak scaling) or one layer split by KV head group (strong scaling)")
+    ap.add_argument("--projection", action="store_true",
+                    help="time the fused query/key projection (Eq. 1) and the estimate that uses its summaries, instead of the bench line")
+    ap.add_argument("--d-model", type=int, default=4096)
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -640,6 +692,8 @@ def main():
         run_fusion_ablation(args, cfg)
     elif args.overlap:
         run_overlap(args, cfg)
+    elif args.projection:
+        run_projection(args, cfg)
     else:
         run_ours(args, cfg)
 

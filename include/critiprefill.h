@@ -67,6 +67,8 @@ enum {
   CP_FLAG_FORCE_SPLIT_SCORE = 16,  /* estimate: take the two-kernel score path (tensor-core log-sum-exps + exact logits of
                                       the visible blocks) whatever the size of the score map; without the flag it is used
                                       from a few million scores up, where it is faster (16-bit inputs, head_dim 128) */
+  CP_FLAG_SUMMARIES_READY = 32,    /* estimate: the workspace already holds the representatives of these Q and K, written by
+                                      critiprefill_project_qk with the same parameters: skip the pass over Q and K */
   CP_FLAG_SHARED_GROUP_LISTS = 8   /* select: one list per KV group instead of one per query head -- the g query
                                       heads of a KV head all receive the list selected from the element-wise
                                       maximum of their scores (a variant; the paper describes a single head) */
@@ -149,6 +151,23 @@ size_t critiprefill_static_scratch_bytes(void);
  * Exact (comparisons only). */
 int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32_t* cnt, void* ws,
                         size_t ws_bytes, void* cuda_stream);
+
+/* Eq. 1 for queries and keys, fused with what Algorithm 1 needs from them: Q = W_Q X and K = W_K X on the tensor cores
+ * (16-bit operands, fp32 accumulation), rotary position embedding in fp32 (rotate-half pairing: channel i with channel
+ * i + head_dim/2, angle given by the caller's tables; the paper does not mention it, the models it evaluates apply it
+ * here), results rounded once to the 16-bit dtype and stored -- and, from those stored values, the per-channel max / min
+ * of every query segment and key block (Algorithm 1, lines 3-8) written to `ws`, so that a following
+ * critiprefill_estimate with CP_FLAG_SUMMARIES_READY and the same `p` and `ws` need not read Q and K again.
+ *   X          in   device, [batch, seq_len, d_model] contiguous, dtype as in p (bf16 or fp16)
+ *   Wq, Wk     in   device, [n_q_heads*head_dim, d_model] and [n_kv_heads*head_dim, d_model], row-major
+ *   rope_cos, rope_sin  in  device, nullable together: [seq_len, head_dim/2] fp32; NULL = no rotation (Eq. 1 as printed)
+ *   Q_out, K_out  out  device, layouts given by p->q_stride / p->k_stride
+ * Supported: head_dim 128, segment_size % 128 == 0, block_size in {32, 64, 128}, d_model % 64 == 0, seq_len >= 128
+ * (else CP_ERR_UNSUPPORTED).  The representatives are bit-identical to what critiprefill_estimate computes from the
+ * stored Q_out, K_out. */
+int critiprefill_project_qk(const cp_params* p, const void* X, const void* Wq, const void* Wk, const float* rope_cos,
+                            const float* rope_sin, int32_t d_model, void* Q_out, void* K_out, void* ws, size_t ws_bytes,
+                            void* cuda_stream);
 
 /* Query criticality of the LAST token, the decoding-phase use that Section 2.1 describes (the query of the last
  * token against the cached keys).  The paper gives no formula for it; this is Algorithm 1 on a segment that holds

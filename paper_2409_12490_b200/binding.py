@@ -23,12 +23,13 @@ FLAG_FORCE_SIMT = 2
 FLAG_TEST_WITHHOLD_V = 4
 FLAG_SHARED_GROUP_LISTS = 8
 FLAG_FORCE_SPLIT_SCORE = 16
+FLAG_SUMMARIES_READY = 32
 
 EXPORTS = (
     "critiprefill_workspace_bytes", "critiprefill_estimate", "critiprefill_select",
     "critiprefill_attention", "critiprefill_dense_attention", "critiprefill_device_status",
     "critiprefill_estimate_static", "critiprefill_static_scratch_bytes",
-    "critiprefill_decode_estimate", "critiprefill_decode_select",
+    "critiprefill_decode_estimate", "critiprefill_decode_select", "critiprefill_project_qk",
     "critiprefill_status_string",
 )
 
@@ -74,6 +75,7 @@ def load_library() -> ctypes.CDLL:
         lib.critiprefill_estimate_static.argtypes = [PP, P, P, P, P, P]
         lib.critiprefill_decode_estimate.argtypes = [PP, P, P, P, P, SZ, P]
         lib.critiprefill_decode_select.argtypes = [PP, P, P, P, P, SZ, P]
+        lib.critiprefill_project_qk.argtypes = [PP, P, P, P, P, P, ctypes.c_int32, P, P, P, SZ, P]
         lib.critiprefill_static_scratch_bytes.argtypes = []
         lib.critiprefill_status_string.argtypes = [ctypes.c_int]
         lib.critiprefill_status_string.restype = ctypes.c_char_p
@@ -209,6 +211,22 @@ def select(prob: Problem, S, ws, idx=None, cnt=None):
     _check(load_library().critiprefill_select(ctypes.byref(p), _ptr(S), _ptr(idx), _ptr(cnt), _ptr(ws), ws.numel(),
                                               _stream()), "critiprefill_select")
     return idx, cnt
+
+
+def project_qk(prob: Problem, X, Wq, Wk, ws, rope_cos=None, rope_sin=None, Q_out=None, K_out=None):
+    """critiprefill_project_qk: Q = W_Q X, K = W_K X (Eq. 1) with rotary embedding; also leaves the representatives of
+    Algorithm 1 in `ws` (follow with estimate(..., flags |= FLAG_SUMMARIES_READY)).  Returns (Q [B,Hq,n,d], K [B,Hkv,n,d])."""
+    B, n, d_model = X.shape
+    assert X.is_contiguous() and Wq.is_contiguous() and Wk.is_contiguous()
+    if Q_out is None:
+        Q_out = torch.empty((B, prob.n_q_heads, n, prob.head_dim), dtype=X.dtype, device=X.device)
+    if K_out is None:
+        K_out = torch.empty((B, prob.n_kv_heads, n, prob.head_dim), dtype=X.dtype, device=X.device)
+    p = prob.params(Q=Q_out, K=K_out)
+    _check(load_library().critiprefill_project_qk(ctypes.byref(p), _ptr(X), _ptr(Wq), _ptr(Wk), _ptr(rope_cos), _ptr(rope_sin),
+                                                  int(d_model), _ptr(Q_out), _ptr(K_out), _ptr(ws), ws.numel(), _stream()),
+           "critiprefill_project_qk")
+    return Q_out, K_out
 
 
 def decode_estimate(prob: Problem, q_last, K, ws, S_out=None) -> torch.Tensor:

@@ -68,13 +68,14 @@ int critiprefill_estimate(const cp_params* p, const void* Q, const void* K, cons
   Dims m;
   int rc = validate(p, &m);
   if (rc != CP_OK) return rc;
-  if (!Q || !K || !S_out) return CP_ERR_NULL;
-  if (!aligned16(Q) || !aligned16(K) || S_out == S_prev) return CP_ERR_SHAPE;
+  const bool ready = (p->flags & CP_FLAG_SUMMARIES_READY) != 0;   // ws already holds the representatives (critiprefill_project_qk)
+  if ((!ready && (!Q || !K)) || !S_out) return CP_ERR_NULL;
+  if ((!ready && (!aligned16(Q) || !aligned16(K))) || S_out == S_prev) return CP_ERR_SHAPE;
   if (S_prev != nullptr && !(p->alpha >= 0.0f && p->alpha <= 1.0f)) return CP_ERR_SHAPE;   // line 14 is a convex combination (NaN fails too)
   if (m.n2 > kMaxBlocksN2) return CP_ERR_UNSUPPORTED;
   if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  if ((rc = launch_summarize(*p, m, Q, K, static_cast<char*>(ws), s)) != CP_OK) return rc;
+  if (!ready && (rc = launch_summarize(*p, m, Q, K, static_cast<char*>(ws), s)) != CP_OK) return rc;
   return launch_score(*p, m, static_cast<char*>(ws), S_prev, S_out, s);
 }
 
@@ -86,6 +87,21 @@ int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32
   if (!S || !idx || !cnt) return CP_ERR_NULL;
   if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
   return launch_select(*p, m, S, idx, cnt, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int critiprefill_project_qk(const cp_params* p, const void* X, const void* Wq, const void* Wk, const float* rope_cos,
+                            const float* rope_sin, int32_t d_model, void* Q_out, void* K_out, void* ws, size_t ws_bytes,
+                            void* cuda_stream) {
+  Dims m;
+  int rc = validate(p, &m);
+  if (rc != CP_OK) return rc;
+  if (!X || !Wq || !Wk || !Q_out || !K_out || ((rope_cos == nullptr) != (rope_sin == nullptr))) return CP_ERR_NULL;
+  if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Q_out) || !aligned16(K_out) || !aligned16(rope_cos) ||
+      !aligned16(rope_sin) || d_model <= 0)
+    return CP_ERR_SHAPE;
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  return launch_project(*p, m, X, Wq, Wk, rope_cos, rope_sin, d_model, Q_out, K_out, static_cast<char*>(ws),
+                        static_cast<cudaStream_t>(cuda_stream));
 }
 
 int critiprefill_decode_estimate(const cp_params* p, const void* q_last, const void* K, double* S_out, void* ws,
