@@ -92,12 +92,22 @@ struct Args {
   unsigned int* work_counter;   // next unit to hand out (zeroed by the host before the launch)
 };
 
-// Optional cycle trace (compiled only with -DCP_TRACE, never in the product build): one CTA
-// records clock64() stamps into the workspace behind the status block.
+// Optional event trace (compiled only with -DCP_TRACE, never in the product build): in CTA 0 the first softmax warp of
+// each query tile, the producer and the MMA warp each append (clock, tag) pairs for units 4..7 to a region of their own
+// in the workspace behind the status block (plain stores, a counter in a register: the traced warp never waits).
 #ifdef CP_TRACE
-#define CP_STAMP(cond, slot) do { if (cond) reinterpret_cast<long long*>(reinterpret_cast<char*>(a.st) + 256)[slot] = clock64(); } while (0)
+__device__ __forceinline__ unsigned long long trace_clock() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%clock64;" : "=l"(t) :: "memory");
+  return t;
+}
+#define CP_EV_DECL unsigned ev_n = 0
+#define CP_EV(cond, q, tag) do { if ((cond) && blockIdx.x == 0 && (q) >= 4u && (q) < 8u && ev_n < 1024u) { \
+    reinterpret_cast<unsigned long long*>(reinterpret_cast<char*>(a.st) + 4096)[((tag) / 100 - 1 + ((tag) >= 110 && (tag) < 120 ? 3 : 0)) * 1024 + ev_n++] = \
+        (trace_clock() << 12) | (unsigned long long)(tag); } } while (0)
 #else
-#define CP_STAMP(cond, slot) do { } while (0)
+#define CP_EV_DECL
+#define CP_EV(cond, q, tag) do { } while (0)
 #endif
 
 // bounded wait on one of this kernel's barriers (the CTA's abort flag lives in the barrier block)
@@ -256,6 +266,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
   const uint32_t tO = tm + lane_off + 256 + which * 128;
   const int row = warp_in_wg * 32 + lane;
   const float c = a.sm_scale * 1.4426950408889634f;   // logits -> log2 units
+  CP_EV_DECL;
   uint32_t n_tiles = 0;                               // S tiles consumed so far (all units)
   uint32_t n_units = 0;                               // units finished so far
 
@@ -280,15 +291,13 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     float m_run = -CUDART_INF, l_run = 0.f;
 
     for (int jt = 0; jt < my_tiles; ++jt, ++n_tiles) {
-      [[maybe_unused]] const bool tr = blockIdx.x == 0 && q == 0 && warp_in_wg == 0 && lane == 0 && jt < 64;
-      CP_STAMP(tr, which * 1024 + jt * 8 + 0);
+      CP_EV(warp_in_wg == 0 && lane == 0, q, 100 + which * 10 + 0);          // waiting for S
       if (!mbar_wait(&bars->s_full[which], n_tiles & 1, bars, a.st, 10 + which)) return;
-      CP_STAMP(tr, which * 1024 + jt * 8 + 1);
+      CP_EV(warp_in_wg == 0 && lane == 0, q, 100 + which * 10 + 1);          // S ready
       tc_fence_after();
       uint32_t sv[128];
       tmem_ld128(tS, sv);
       tmem_wait_ld();
-      CP_STAMP(tr, which * 1024 + jt * 8 + 2);
       float* s = reinterpret_cast<float*>(sv);
 
       int kind = kMaskNone, cols = kTile;
@@ -350,7 +359,6 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
           tmem_st32(tO + q * 32, ov);
         }
       }
-      CP_STAMP(tr, which * 1024 + jt * 8 + 3);
       const float neg_mc = (m_run == -CUDART_INF) ? 0.f : -m_run * c;   // a row that has not seen a key yet (generic lists only): exp2(-inf) = 0
       const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
       float2 sum2 = make_float2(0.f, 0.f);
@@ -377,17 +385,17 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
         }
       }
       l_run += sum2.x + sum2.y;
-      CP_STAMP(tr, which * 1024 + jt * 8 + 4);
       tmem_st64(tS, pk);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->p_full[which]);
-      CP_STAMP(tr, which * 1024 + jt * 8 + 5);
+      CP_EV(warp_in_wg == 0 && lane == 0, q, 100 + which * 10 + 2);          // P handed over
     }
 
     // epilogue: O / l -> bf16 -> global.  The next unit's first PV cannot start before this
     // thread signals its next P, so O is not overwritten while it is being read.
     if (!mbar_wait(&bars->o_done[which], n_units & 1, bars, a.st, 20 + which)) return;
+    CP_EV(warp_in_wg == 0 && lane == 0, q, 100 + which * 10 + 3);            // O complete
     ++n_units;
     tc_fence_after();
     const int t = u.q_tok + which * kTile + row;
@@ -416,6 +424,7 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
     }
     if (a.lse != nullptr && t < a.n)
       a.lse[((long long)u.b * a.Hq + u.h) * a.n + t] = m_run * a.sm_scale + __logf(l_run);
+    CP_EV(warp_in_wg == 0 && lane == 0, q, 100 + which * 10 + 4);            // epilogue done
   }
 }
 
@@ -424,6 +433,7 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
                                               const CUtensorMap* tmKb, const CUtensorMap* tmVb,
                                               const CUtensorMap* tmKt, const CUtensorMap* tmVt, int lane) {
   const int bpt = kTile / a.blk;
+  CP_EV_DECL;
   uint32_t item = 0;      // K/V tiles issued so far (all units): item i lives in slot i % kSlots
   uint32_t n_units = 0;
   // One unit of look-ahead: unit q+1 is drawn, checked and published before the loads of unit q
@@ -437,10 +447,13 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
     // pay at every unit); it tells them through the CTA's abort flag, which their waits poll.
     if (stop_requested(a, bars)) { bars->abort_flag = 1; return; }
     const Unit u_cur = u;
+    CP_EV(lane == 0, q, 300);                                                // producer starts unit q
     if (!publish_unit(a, bars, q + 1, lane, &x, &u)) return;
+    CP_EV(lane == 0, q, 301);                                                // unit q+1 published
     if (u_cur.cnt == kBadList || u_cur.cnt == kEmptyUnit || u_cur.cnt == kZeroUnit) continue;
     // Q tiles: the buffer is free once every QK^T of the previous unit has completed
     if (n_units > 0 && !mbar_wait(&bars->q_empty, (n_units - 1) & 1, bars, a.st, 31)) return;
+    CP_EV(lane == 0, q, 302);                                                // Q buffer free: Q loads go out
     if (lane == 0) {
       const int nq = u_cur.nB ? 2 : 1;
       mbar_expect_tx(&bars->q_full, nq * kTileBytes);
@@ -453,6 +466,7 @@ __device__ __forceinline__ void producer_role(const Args& a, Bars* bars, uint32_
     for (int it = 0; it < 2 * u_cur.T; ++it, ++item) {   // 2*jt = K tile jt, 2*jt+1 = V tile jt
       const uint32_t slot = item % kSlots, use = item / kSlots;
       if (use > 0 && !mbar_wait(&bars->kv_empty[slot], (use - 1) & 1, bars, a.st, 30)) return;
+      CP_EV(lane == 0, q, 310 + (it < 40 ? it : 40));                        // slot free: K/V item `it` goes out
       if (lane == 0 && !(a.withhold_v && (it & 1))) {
         const int jt = it >> 1;
         const bool is_v = it & 1;
@@ -503,6 +517,7 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
   const uint32_t tm = __shfl_sync(0xffffffffu, bars->tmem_base, 0);
   const uint32_t tS[2] = {tm, tm + 128}, tO[2] = {tm + 256, tm + 384};
   const uint32_t qA = smem_base + kSmemQ, qB = qA + kTileBytes;
+  CP_EV_DECL;
   uint32_t item0 = 0;                 // first K/V item of the current unit
   uint32_t nA = 0, nB = 0;            // P tiles consumed so far per query tile (all units)
   uint32_t n_units = 0;
@@ -513,12 +528,16 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
   for (uint32_t q = 0;; ++q) {
     int x;
     Unit u;
+    CP_EV(lane == 0, q, 205);                                                // asks for the unit
     if (!receive_unit(a, bars, q, lane, &x, &u) || x >= a.n_units || bars->abort_flag) return;
     if (u.cnt == kBadList || u.cnt == kEmptyUnit || u.cnt == kZeroUnit) continue;
     const int T = u.T, TA = u.nA;
     const bool hasB = u.nB > 0;
+    CP_EV(lane == 0, q, 200);                                                // unit received
     if (!mbar_wait(&bars->q_full, n_units & 1, bars, a.st, 41)) return;
+    CP_EV(lane == 0, q, 201);                                                // Q ready
     if (!full_wait(item0)) return;
+    CP_EV(lane == 0, q, 202);                                                // K0 ready
     tc_fence_after();
     issue_qk<kF16>(tS[0], qA, slot_addr(item0)); umma_commit(&bars->s_full[0]);
     if (hasB) { issue_qk<kF16>(tS[1], qB, slot_addr(item0)); umma_commit(&bars->s_full[1]); }
@@ -530,22 +549,20 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
       if (has_next && !full_wait(ik)) return;
       if (!full_wait(iv)) return;
       const uint32_t v_smem = slot_addr(iv), kn_smem = slot_addr(ik);
-      [[maybe_unused]] const bool tr = blockIdx.x == 0 && q == 0 && lane == 0 && jt < 64;
-      CP_STAMP(tr, 2048 + jt * 8 + 0);
       if (jt < TA) {
         if (!mbar_wait(&bars->p_full[0], nA & 1, bars, a.st, 42)) return;
+        CP_EV(lane == 0, q, 210);                                            // P_A ready
         ++nA;
-        CP_STAMP(tr, 2048 + jt * 8 + 1);
         tc_fence_after();
         issue_pv<kF16>(tO[0], tS[0], v_smem, jt > 0);
         if (jt + 1 < TA) { issue_qk<kF16>(tS[0], qA, kn_smem); umma_commit(&bars->s_full[0]); }
         else umma_commit(&bars->o_done[0]);
       }
-      CP_STAMP(tr, 2048 + jt * 8 + 2);
       if (hasB) {
+        CP_EV(lane == 0, q, 211);                                            // group A issued
         if (!mbar_wait(&bars->p_full[1], nB & 1, bars, a.st, 43)) return;
+        CP_EV(lane == 0, q, 212);                                            // P_B ready
         ++nB;
-        CP_STAMP(tr, 2048 + jt * 8 + 3);
         tc_fence_after();
         issue_pv<kF16>(tO[1], tS[1], v_smem, jt > 0);
       }
@@ -557,7 +574,7 @@ __device__ __forceinline__ void mma_role(const Args& a, Bars* bars, uint32_t sme
       } else if (hasB) {
         umma_commit(&bars->o_done[1]);
       }
-      CP_STAMP(tr, 2048 + jt * 8 + 4);
+      CP_EV(lane == 0, q, 213);                                              // tile step issued
     }
     item0 += 2 * T;
     ++n_units;
