@@ -214,6 +214,30 @@ int critiprefill_dense_attention(const cp_params* p, const void* Q, const void* 
                                  void* O, float* lse, void* ws, size_t ws_bytes,
                                  void* cuda_stream);
 
+/* A packed batch of sequences of different lengths: one layer of the hot path (Algorithm 1, Algorithm 2 line 8,
+ * Algorithm 2 lines 6-13) for each sequence.  The paper describes a single sequence; here every sequence is a problem
+ * of its own: its segments and blocks are counted from its first token, its block indices are relative to that token,
+ * and no query sees a key of another sequence.
+ *   p           batch must be 1; seq_len = the LONGEST sequence (it sizes `ws`); the strides' batch entry is ignored,
+ *               their head and token entries describe the packed tensors [total_tokens, heads, head_dim]
+ *   cu_seqlens  in  HOST, n_seqs + 1 entries: 0, len_0, len_0 + len_1, ...; strictly increasing; len_i <= p->seq_len.
+ *               Sequence i holds packed tokens [cu_seqlens[i], cu_seqlens[i+1])
+ *   Q, K, V     in  device, packed;  O out device, packed;  lse out device, nullable, [Hq] x packed token:
+ *               sequence i's part is the [Hq, len_i] array that starts at element Hq * cu_seqlens[i]
+ *   S_prev      in  device, nullable; S_out, idx, cnt  out device: the per-sequence arrays of critiprefill_estimate /
+ *               critiprefill_select ([Hq,n1_i,n2_i] fp64, [Hq,n1_i,k] int32, [Hq,n1_i] int32 with n1_i, n2_i from
+ *               len_i) stored one after another in sequence order; critiprefill_varlen_sizes gives the totals
+ * The sequences run one after another on `cuda_stream` through the same kernels as the single-sequence calls, so each
+ * sequence's results are those of critiprefill_estimate + _select + _attention on its slice, bit for bit.
+ * Errors: CP_ERR_SHAPE for a bad cu_seqlens or batch != 1; otherwise as the single-sequence calls. */
+int critiprefill_prefill_varlen(const cp_params* p, const int32_t* cu_seqlens, int32_t n_seqs, const void* Q,
+                                const void* K, const void* V, const double* S_prev, double* S_out, int32_t* idx,
+                                int32_t* cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Element counts of the packed S (fp64), idx and cnt (int32) arrays of critiprefill_prefill_varlen.  Host pointers. */
+int critiprefill_varlen_sizes(const cp_params* p, const int32_t* cu_seqlens, int32_t n_seqs, int64_t* s_elems,
+                              int64_t* idx_elems, int64_t* cnt_elems);
+
 /* Synchronises `cuda_stream`, copies the device status word (a cp_status: CP_OK, CP_ERR_TIMEOUT
  * or CP_ERR_BOUNDS; sticky until the caller zeroes the status block) to *status_out (host). */
 int critiprefill_device_status(const void* ws, int32_t* status_out, void* cuda_stream);

@@ -17,6 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcritiprefill.so")
 
 CP_OK = 0
+CP_ERR_NULL, CP_ERR_SHAPE = 1, 2
 CP_BF16, CP_F32, CP_F16 = 0, 1, 2
 FLAG_MASK_BEFORE_SOFTMAX = 1
 FLAG_FORCE_SIMT = 2
@@ -30,6 +31,7 @@ EXPORTS = (
     "critiprefill_attention", "critiprefill_dense_attention", "critiprefill_device_status",
     "critiprefill_estimate_static", "critiprefill_static_scratch_bytes",
     "critiprefill_decode_estimate", "critiprefill_decode_select", "critiprefill_project_qk",
+    "critiprefill_prefill_varlen", "critiprefill_varlen_sizes",
     "critiprefill_status_string",
 )
 
@@ -76,6 +78,9 @@ def load_library() -> ctypes.CDLL:
         lib.critiprefill_decode_estimate.argtypes = [PP, P, P, P, P, SZ, P]
         lib.critiprefill_decode_select.argtypes = [PP, P, P, P, P, SZ, P]
         lib.critiprefill_project_qk.argtypes = [PP, P, P, P, P, P, ctypes.c_int32, P, P, P, SZ, P]
+        lib.critiprefill_prefill_varlen.argtypes = [PP, P, ctypes.c_int32, P, P, P, P, P, P, P, P, P, P, SZ, P]
+        I64P = ctypes.POINTER(ctypes.c_int64)
+        lib.critiprefill_varlen_sizes.argtypes = [PP, P, ctypes.c_int32, I64P, I64P, I64P]
         lib.critiprefill_static_scratch_bytes.argtypes = []
         lib.critiprefill_status_string.argtypes = [ctypes.c_int]
         lib.critiprefill_status_string.restype = ctypes.c_char_p
@@ -280,6 +285,51 @@ def device_status(ws) -> int:
     out = ctypes.c_int32(0)
     _check(load_library().critiprefill_device_status(_ptr(ws), ctypes.byref(out), _stream()), "critiprefill_device_status")
     return int(out.value)
+
+
+def _packed_strides(t: torch.Tensor):
+    """Strides of a packed [heads, total_tokens, d] view as (batch: unused, head, token)."""
+    assert t.dim() == 3 and t.stride(2) == 1
+    return (ctypes.c_int64 * 3)(0, t.stride(0), t.stride(1))
+
+
+def prefill_varlen(prob: Problem, cu_seqlens, Q, K, V, ws, S_prev=None, want_lse=False):
+    """critiprefill_prefill_varlen: one layer for every sequence of a packed batch.
+
+    Q [Hq, total, d], K and V [Hkv, total, d] (any head / token strides, e.g. views of [total, H, d] storage);
+    cu_seqlens: host integers 0, len_0, len_0 + len_1, ...; prob.batch = 1 and prob.seq_len = the longest sequence.
+    Returns (O, S, idx, cnt, S_flat[, lse]): O like Q; S, idx, cnt are lists of per-sequence views ([Hq,n1_i,n2_i]
+    fp64, [Hq,n1_i,k] int32, [Hq,n1_i] int32) of the packed arrays the call fills; S_flat is the packed score array
+    itself, which is what the next layer's call takes as S_prev; lse is [Hq * total] fp32, sequence i's [Hq, len_i]
+    part starting at Hq * cu_seqlens[i]."""
+    lib = load_library()
+    cu = (ctypes.c_int32 * len(cu_seqlens))(*[int(c) for c in cu_seqlens])
+    n_seqs = len(cu_seqlens) - 1
+    p = prob.params()
+    p.q_stride, p.k_stride, p.v_stride = _packed_strides(Q), _packed_strides(K), _packed_strides(V)
+    O = torch.empty_like(Q)
+    p.o_stride = _packed_strides(O)
+    sizes = [ctypes.c_int64(0) for _ in range(3)]
+    _check(lib.critiprefill_varlen_sizes(ctypes.byref(p), cu, n_seqs, *[ctypes.byref(s) for s in sizes]),
+           "critiprefill_varlen_sizes")
+    S_flat = torch.empty(sizes[0].value, dtype=torch.float64, device=Q.device)
+    idx_flat = torch.empty(sizes[1].value, dtype=torch.int32, device=Q.device)
+    cnt_flat = torch.empty(sizes[2].value, dtype=torch.int32, device=Q.device)
+    lse = torch.empty((prob.n_q_heads * Q.shape[1],), dtype=torch.float32, device=Q.device) if want_lse else None
+    _check(lib.critiprefill_prefill_varlen(ctypes.byref(p), cu, n_seqs, _ptr(Q), _ptr(K), _ptr(V), _ptr(S_prev), _ptr(S_flat),
+                                           _ptr(idx_flat), _ptr(cnt_flat), _ptr(O), _ptr(lse), _ptr(ws), ws.numel(), _stream()),
+           "critiprefill_prefill_varlen")
+    S, idx, cnt = [], [], []
+    so = io = co = 0
+    H, k = prob.n_q_heads, prob.budget_blocks
+    for a, b in zip(cu_seqlens[:-1], cu_seqlens[1:]):
+        n = int(b) - int(a)
+        n1, n2 = -(-n // prob.segment_size), -(-n // prob.block_size)
+        S.append(S_flat[so:so + H * n1 * n2].view(H, n1, n2)); so += H * n1 * n2
+        idx.append(idx_flat[io:io + H * n1 * k].view(H, n1, k)); io += H * n1 * k
+        cnt.append(cnt_flat[co:co + H * n1].view(H, n1)); co += H * n1
+    out = (O, S, idx, cnt, S_flat)
+    return out + (lse,) if want_lse else out
 
 
 def prefill_layer(prob: Problem, Q, K, V, ws, S_prev=None):

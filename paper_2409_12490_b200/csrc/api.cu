@@ -1,6 +1,8 @@
 // The C ABI (include/critiprefill.h): argument validation and kernel dispatch.
 #include "cp_common.cuh"
 
+#include <vector>
+
 namespace {
 
 using namespace cp;
@@ -150,6 +152,75 @@ int critiprefill_attention(const cp_params* p, const void* Q, const void* K, con
 int critiprefill_dense_attention(const cp_params* p, const void* Q, const void* K, const void* V, void* O,
                                  float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
   return attention_common(p, Q, K, V, nullptr, nullptr, O, lse, ws, ws_bytes, cuda_stream, true);
+}
+
+namespace {
+// cu_seqlens checked, and the packed offsets of sequence i's S / idx / cnt arrays (in elements)
+struct SeqSlot { int64_t s, idx, cnt; int len; };
+int varlen_walk(const cp_params* p, const int32_t* cu, int32_t n_seqs, std::vector<SeqSlot>* slots, SeqSlot* total) {
+  if (p == nullptr || cu == nullptr) return CP_ERR_NULL;
+  if (n_seqs <= 0 || cu[0] != 0 || p->batch != 1 || p->segment_size <= 0 || p->block_size <= 0 || p->budget_blocks <= 0 ||
+      p->n_q_heads <= 0)
+    return CP_ERR_SHAPE;
+  SeqSlot at{0, 0, 0, 0};
+  for (int i = 0; i < n_seqs; ++i) {
+    const int64_t len = int64_t(cu[i + 1]) - cu[i];
+    if (len <= 0 || len > p->seq_len) return CP_ERR_SHAPE;
+    const int64_t n1 = (len + p->segment_size - 1) / p->segment_size, n2 = (len + p->block_size - 1) / p->block_size;
+    at.len = int(len);
+    if (slots != nullptr) slots->push_back(at);
+    at.s += int64_t(p->n_q_heads) * n1 * n2;
+    at.idx += int64_t(p->n_q_heads) * n1 * p->budget_blocks;
+    at.cnt += int64_t(p->n_q_heads) * n1;
+  }
+  *total = at;
+  return CP_OK;
+}
+}  // namespace
+
+int critiprefill_varlen_sizes(const cp_params* p, const int32_t* cu_seqlens, int32_t n_seqs, int64_t* s_elems,
+                              int64_t* idx_elems, int64_t* cnt_elems) {
+  if (!s_elems || !idx_elems || !cnt_elems) return CP_ERR_NULL;
+  SeqSlot total;
+  const int rc = varlen_walk(p, cu_seqlens, n_seqs, nullptr, &total);
+  if (rc != CP_OK) return rc;
+  *s_elems = total.s; *idx_elems = total.idx; *cnt_elems = total.cnt;
+  return CP_OK;
+}
+
+int critiprefill_prefill_varlen(const cp_params* p, const int32_t* cu_seqlens, int32_t n_seqs, const void* Q,
+                                const void* K, const void* V, const double* S_prev, double* S_out, int32_t* idx,
+                                int32_t* cnt, void* O, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
+  std::vector<SeqSlot> slots;
+  SeqSlot total;
+  int rc = varlen_walk(p, cu_seqlens, n_seqs, &slots, &total);
+  if (rc != CP_OK) return rc;
+  Dims m;
+  if ((rc = validate(p, &m)) != CP_OK) return rc;   // the longest sequence: strides, dtype, head geometry, budget
+  if (!Q || !K || !V || !O || !S_out || !idx || !cnt) return CP_ERR_NULL;
+  if (p->flags & CP_FLAG_SUMMARIES_READY) return CP_ERR_UNSUPPORTED;   // the workspace holds one sequence's representatives at a time
+  if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
+  auto at = [&](const void* base, int64_t token, const int64_t* stride) {
+    return static_cast<const char*>(base) + token * stride[2] * m.es;
+  };
+  for (int i = 0; i < n_seqs; ++i) {
+    cp_params q = *p;
+    q.seq_len = slots[i].len;
+    const int64_t t0 = cu_seqlens[i];
+    const void* Qi = at(Q, t0, p->q_stride);
+    const void* Ki = at(K, t0, p->k_stride);
+    const void* Vi = at(V, t0, p->v_stride);
+    void* Oi = const_cast<char*>(at(O, t0, p->o_stride));
+    double* Si = S_out + slots[i].s;
+    int32_t* idx_i = idx + slots[i].idx;
+    int32_t* cnt_i = cnt + slots[i].cnt;
+    if ((rc = critiprefill_estimate(&q, Qi, Ki, S_prev ? S_prev + slots[i].s : nullptr, Si, ws, ws_bytes, cuda_stream)) != CP_OK) return rc;
+    if ((rc = critiprefill_select(&q, Si, idx_i, cnt_i, ws, ws_bytes, cuda_stream)) != CP_OK) return rc;
+    if ((rc = critiprefill_attention(&q, Qi, Ki, Vi, idx_i, cnt_i, Oi, lse ? lse + int64_t(p->n_q_heads) * t0 : nullptr, ws, ws_bytes,
+                                     cuda_stream)) != CP_OK)
+      return rc;
+  }
+  return CP_OK;
 }
 
 int critiprefill_device_status(const void* ws, int32_t* status_out, void* cuda_stream) {
