@@ -1,4 +1,4 @@
-"""Oracle: the query / key projections of Eq. 1 with rotary position embedding, fp64, plain numpy.
+"""Oracle: the query / key / value projections of Eq. 1, rotary position embedding on Q and K, fp64, plain numpy.
 
 TEST INFRASTRUCTURE -- checks the fused projection kernel; not part of the product path.
 
@@ -11,7 +11,8 @@ angle whose cosine / sine the caller tabulates per token, cos[t,i], sin[t,i]:
 The paper does not mention position embeddings; the models it evaluates (Llama3, Yi) apply this rotation to Q and K
 right after the projection, which is why the fused kernel carries it.  (cos = 1, sin = 0 gives Eq. 1 as printed.)
 
-Pins (tests/test_oracle_projection.py): the matrix product against explicit loops; the rotation against complex
+V = W_V X is the plain product.
+Pins (tests/test_oracle_projection.py): the matrix products against explicit loops; the rotation against complex
 multiplication (x[i] + 1j x[i+d/2]) * exp(1j theta), norm preservation, and the identity for theta = 0.
 """
 from __future__ import annotations
@@ -48,6 +49,19 @@ def project_qk(X, Wq, Wk, head_dim: int, cos=None, sin=None):
             P = rope(P, _f64(cos), _f64(sin))
         out.append(P)
     return out[0], out[1]
+
+
+def project_v(X, Wv, head_dim: int):
+    """V = W_V X of Eq. 1: X [B,n,d_model], Wv [Hkv*d, d_model] -> V [B,Hkv,n,d] in fp64 (not rounded).  Values carry no
+    position embedding and Algorithm 1 takes nothing from them, so this is the matrix product alone."""
+    X, Wv = _f64(X), _f64(Wv)
+    B, n, _ = X.shape
+    H = Wv.shape[0] // head_dim
+    V = np.empty((B, H, n, head_dim), dtype=np.float64)
+    for b in range(B):
+        for h in range(H):
+            V[b, h] = X[b] @ Wv[h * head_dim:(h + 1) * head_dim].T
+    return V
 
 
 def rope_tables(n: int, head_dim: int, theta: float = 500000.0):

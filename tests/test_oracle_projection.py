@@ -1,7 +1,7 @@
 """Pins for oracle/projection.py (Eq. 1 with rotary embedding).  CPU only."""
 import numpy as np
 
-from oracle.projection import project_qk, rope, rope_tables
+from oracle.projection import project_qk, project_v, rope, rope_tables
 
 
 def test_projection_is_the_matrix_product_of_eq_1():
@@ -19,6 +19,23 @@ def test_projection_is_the_matrix_product_of_eq_1():
             for h in range(Hkv):
                 for c in range(d):
                     assert abs(K[b, h, t, c] - sum(Wk[h * d + c, m] * X[b, t, m] for m in range(dm))) < 1e-12
+
+
+def test_value_projection_is_the_matrix_product_of_eq_1():
+    rng = np.random.default_rng(5)
+    B, n, dm, d, Hkv = 2, 4, 5, 3, 2
+    X = rng.standard_normal((B, n, dm))
+    Wv = rng.standard_normal((Hkv * d, dm))
+    V = project_v(X, Wv, d)
+    assert V.shape == (B, Hkv, n, d)
+    for b in range(B):
+        for t in range(n):
+            for h in range(Hkv):
+                for c in range(d):
+                    assert abs(V[b, h, t, c] - sum(Wv[h * d + c, m] * X[b, t, m] for m in range(dm))) < 1e-12
+    # a one-hot X row picks out a column of W_V
+    X1 = np.zeros((1, 1, dm)); X1[0, 0, 2] = 1.0
+    np.testing.assert_array_equal(project_v(X1, Wv, d)[0, :, 0, :].reshape(-1), Wv[:, 2])
 
 
 def test_rotation_is_a_complex_multiplication_and_keeps_norms():
