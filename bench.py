@@ -651,10 +651,23 @@ def run_projection(args, cfg):
     torch.cuda.synchronize()
     assert cp.device_status(ws) == 0
     proj_ms, est_ready_ms, est_plain_ms = (ev[i].elapsed_time(ev[i + 1]) / reps for i in range(3))
+    # the same launch with the value projection of Eq. 1 added
+    Wv = (torch.randn((cfg.n_kv_heads * cfg.head_dim, d_model), generator=g, device=dev) / math.sqrt(d_model)).to(tdt)
+    _, _, V = cp.project_qkv(prob, X, Wq, Wk, Wv, ws, rope_cos=cos, rope_sin=sin, Q_out=Q, K_out=K)
+    torch.cuda.synchronize()
+    ev[0].record()
+    for _ in range(reps):
+        cp.project_qkv(prob, X, Wq, Wk, Wv, ws, rope_cos=cos, rope_sin=sin, Q_out=Q, K_out=K, V_out=V)
+    ev[1].record()
+    torch.cuda.synchronize()
+    qkv_ms = ev[0].elapsed_time(ev[1]) / reps
+    flops_qkv = 2.0 * cfg.batch * cfg.seq_len * d_model * (cfg.n_q_heads + 2 * cfg.n_kv_heads) * cfg.head_dim
     flops = 2.0 * cfg.batch * cfg.seq_len * d_model * (cfg.n_q_heads + cfg.n_kv_heads) * cfg.head_dim
     peaks = load_peaks()
     print(json.dumps({"projection_ms": proj_ms, "gemm_tflops": flops / (proj_ms * 1e-3) / 1e12,
                       "frac_of_bf16_peak": flops / (proj_ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "peak_source": peaks["source"],
+                      "projection_qkv_ms": qkv_ms, "qkv_gemm_tflops": flops_qkv / (qkv_ms * 1e-3) / 1e12,
+                      "qkv_frac_of_bf16_peak": flops_qkv / (qkv_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                       "estimate_ms_summaries_ready": est_ready_ms, "estimate_ms_with_own_pass": est_plain_ms,
                       "scores_identical": same, "d_model": d_model, "config": workload_config(cfg), "data": "synthetic"}))
 

@@ -169,6 +169,13 @@ int critiprefill_project_qk(const cp_params* p, const void* X, const void* Wq, c
                             const float* rope_sin, int32_t d_model, void* Q_out, void* K_out, void* ws, size_t ws_bytes,
                             void* cuda_stream);
 
+/* critiprefill_project_qk with the value projection of Eq. 1 in the same launch: V = W_V X, no rotation, rounded once and
+ * stored with p->v_stride; Algorithm 1 takes nothing from V, so no representatives are formed for it.
+ *   Wv     in   device, [n_kv_heads*head_dim, d_model] row-major;  V_out  out  device.  Both NULL = critiprefill_project_qk. */
+int critiprefill_project_qkv(const cp_params* p, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                             const float* rope_cos, const float* rope_sin, int32_t d_model, void* Q_out, void* K_out,
+                             void* V_out, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /* Query criticality of the LAST token, the decoding-phase use that Section 2.1 describes (the query of the last
  * token against the cached keys).  The paper gives no formula for it; this is Algorithm 1 on a segment that holds
  * that one token: Qmax = Qmin = q, every block is visible, no layer fusion.

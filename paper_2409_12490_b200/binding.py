@@ -31,7 +31,7 @@ EXPORTS = (
     "critiprefill_attention", "critiprefill_dense_attention", "critiprefill_device_status",
     "critiprefill_estimate_static", "critiprefill_static_scratch_bytes",
     "critiprefill_decode_estimate", "critiprefill_decode_select", "critiprefill_project_qk",
-    "critiprefill_prefill_varlen", "critiprefill_varlen_sizes",
+    "critiprefill_prefill_varlen", "critiprefill_varlen_sizes", "critiprefill_project_qkv",
     "critiprefill_status_string",
 )
 
@@ -78,6 +78,7 @@ def load_library() -> ctypes.CDLL:
         lib.critiprefill_decode_estimate.argtypes = [PP, P, P, P, P, SZ, P]
         lib.critiprefill_decode_select.argtypes = [PP, P, P, P, P, SZ, P]
         lib.critiprefill_project_qk.argtypes = [PP, P, P, P, P, P, ctypes.c_int32, P, P, P, SZ, P]
+        lib.critiprefill_project_qkv.argtypes = [PP, P, P, P, P, P, P, ctypes.c_int32, P, P, P, P, SZ, P]
         lib.critiprefill_prefill_varlen.argtypes = [PP, P, ctypes.c_int32, P, P, P, P, P, P, P, P, P, P, SZ, P]
         I64P = ctypes.POINTER(ctypes.c_int64)
         lib.critiprefill_varlen_sizes.argtypes = [PP, P, ctypes.c_int32, I64P, I64P, I64P]
@@ -232,6 +233,22 @@ def project_qk(prob: Problem, X, Wq, Wk, ws, rope_cos=None, rope_sin=None, Q_out
                                                   int(d_model), _ptr(Q_out), _ptr(K_out), _ptr(ws), ws.numel(), _stream()),
            "critiprefill_project_qk")
     return Q_out, K_out
+
+
+def project_qkv(prob: Problem, X, Wq, Wk, Wv, ws, rope_cos=None, rope_sin=None, Q_out=None, K_out=None, V_out=None):
+    """critiprefill_project_qkv: project_qk plus V = W_V X (no rotation) in the same launch.  Returns (Q, K, V)."""
+    B, n, d_model = X.shape
+    assert X.is_contiguous() and Wq.is_contiguous() and Wk.is_contiguous() and Wv.is_contiguous()
+    mk = lambda h: torch.empty((B, h, n, prob.head_dim), dtype=X.dtype, device=X.device)
+    Q_out = mk(prob.n_q_heads) if Q_out is None else Q_out
+    K_out = mk(prob.n_kv_heads) if K_out is None else K_out
+    V_out = mk(prob.n_kv_heads) if V_out is None else V_out
+    p = prob.params(Q=Q_out, K=K_out, V=V_out)
+    _check(load_library().critiprefill_project_qkv(ctypes.byref(p), _ptr(X), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(rope_cos),
+                                                   _ptr(rope_sin), int(d_model), _ptr(Q_out), _ptr(K_out), _ptr(V_out), _ptr(ws),
+                                                   ws.numel(), _stream()),
+           "critiprefill_project_qkv")
+    return Q_out, K_out, V_out
 
 
 def decode_estimate(prob: Problem, q_last, K, ws, S_out=None) -> torch.Tensor:

@@ -91,19 +91,27 @@ int critiprefill_select(const cp_params* p, const double* S, int32_t* idx, int32
   return launch_select(*p, m, S, idx, cnt, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int critiprefill_project_qk(const cp_params* p, const void* X, const void* Wq, const void* Wk, const float* rope_cos,
-                            const float* rope_sin, int32_t d_model, void* Q_out, void* K_out, void* ws, size_t ws_bytes,
-                            void* cuda_stream) {
+int critiprefill_project_qkv(const cp_params* p, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                             const float* rope_cos, const float* rope_sin, int32_t d_model, void* Q_out, void* K_out,
+                             void* V_out, void* ws, size_t ws_bytes, void* cuda_stream) {
   Dims m;
   int rc = validate(p, &m);
   if (rc != CP_OK) return rc;
-  if (!X || !Wq || !Wk || !Q_out || !K_out || ((rope_cos == nullptr) != (rope_sin == nullptr))) return CP_ERR_NULL;
-  if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Q_out) || !aligned16(K_out) || !aligned16(rope_cos) ||
-      !aligned16(rope_sin) || d_model <= 0)
+  if (!X || !Wq || !Wk || !Q_out || !K_out || ((rope_cos == nullptr) != (rope_sin == nullptr)) || ((Wv == nullptr) != (V_out == nullptr)))
+    return CP_ERR_NULL;
+  if (!aligned16(X) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(Q_out) || !aligned16(K_out) ||
+      !aligned16(V_out) || !aligned16(rope_cos) || !aligned16(rope_sin) || d_model <= 0)
     return CP_ERR_SHAPE;
   if ((rc = check_ws(m, ws, ws_bytes)) != CP_OK) return rc;
-  return launch_project(*p, m, X, Wq, Wk, rope_cos, rope_sin, d_model, Q_out, K_out, static_cast<char*>(ws),
+  return launch_project(*p, m, X, Wq, Wk, Wv, rope_cos, rope_sin, d_model, Q_out, K_out, V_out, static_cast<char*>(ws),
                         static_cast<cudaStream_t>(cuda_stream));
+}
+
+int critiprefill_project_qk(const cp_params* p, const void* X, const void* Wq, const void* Wk, const float* rope_cos,
+                            const float* rope_sin, int32_t d_model, void* Q_out, void* K_out, void* ws, size_t ws_bytes,
+                            void* cuda_stream) {
+  return critiprefill_project_qkv(p, X, Wq, Wk, nullptr, rope_cos, rope_sin, d_model, Q_out, K_out, nullptr, ws, ws_bytes,
+                                  cuda_stream);
 }
 
 int critiprefill_decode_estimate(const cp_params* p, const void* q_last, const void* K, double* S_out, void* ws,

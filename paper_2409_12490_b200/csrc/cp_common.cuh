@@ -78,8 +78,8 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
                            const void* V, const int32_t* idx, const int32_t* cnt, void* O,
                            float* lse, DeviceStatus* st, bool dense, cudaStream_t s);
 bool sm100_path_applies(const cp_params& p, const Dims& m);
-int launch_project(const cp_params& p, const Dims& m, const void* X, const void* Wq, const void* Wk, const float* cosT,
-                   const float* sinT, int d_model, void* Q, void* K, char* ws, cudaStream_t s);
+int launch_project(const cp_params& p, const Dims& m, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                   const float* cosT, const float* sinT, int d_model, void* Q, void* K, void* V, char* ws, cudaStream_t st);
 
 inline int check_launch() { return cudaGetLastError() == cudaSuccess ? CP_OK : CP_ERR_CUDA; }
 

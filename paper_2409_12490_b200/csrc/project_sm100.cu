@@ -34,13 +34,13 @@ struct ProjBars {
 };
 
 struct ProjArgs {
-  uint16_t *Q, *K;                            // outputs, 16-bit elements
-  int64_t qsb, qsh, qst, ksb, ksh, kst;       // element strides (batch, head, token)
+  uint16_t *Q, *K, *V;                        // outputs, 16-bit elements (V nullable: no value projection)
+  int64_t qsb, qsh, qst, ksb, ksh, kst, vsb, vsh, vst;   // element strides (batch, head, token)
   const float *cosT, *sinT;                   // [n, 64] fp32, nullable together: no rotation
   uint16_t *Qmax, *Qmin, *Kmax, *Kmin;        // summaries in the workspace
   float* kabs;
   DeviceStatus* st;
-  int B, Hq, Hkv, n, seg, blk, n1, n2, d_model;
+  int B, Hq, Hkv, Hv, n, seg, blk, n1, n2, d_model;   // Hv = Hkv when values are projected too, else 0
   long long n_units;
 };
 
@@ -55,7 +55,7 @@ __device__ __forceinline__ void bar_sync_epilogue() { asm volatile("bar.sync 1, 
 template <bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWq,
-                     const __grid_constant__ CUtensorMap tmWk, const ProjArgs a) {
+                     const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmWv, const ProjArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t smem_base = (raw + 1023u) & ~1023u;
@@ -71,19 +71,25 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 4 && lane == 0) { prefetch_tmap(&tmX); prefetch_tmap(&tmWq); prefetch_tmap(&tmWk); }
+  if (warp == 4 && lane == 0) { prefetch_tmap(&tmX); prefetch_tmap(&tmWq); prefetch_tmap(&tmWk); prefetch_tmap(&tmWv); }
   if (warp == 5) { tmem_alloc(&bars->tmem_base, 512); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tm = bars->tmem_base;
 
-  const int H = a.Hq + a.Hkv;
+  const int Hqk = a.Hq + a.Hkv;            // heads in the order query, key, value
+  const long long n_qk_units = (long long)a.B * Hqk * a.n1;
   const int tiles_per_seg = a.seg / kTileM;
   const int n_kb = a.d_model / kKB;
-  // unit -> (segment j, batch b, head hh); heads of one segment are adjacent so that its X rows stay in L2
+  // unit -> (segment j, batch b, head hh); heads of one segment are adjacent so that its X rows stay in L2.  The value
+  // heads follow in a pass of their own after all query / key units: with all three weight matrices live at once
+  // the weights and the X tiles in flight no longer fit the L2 share of a die and every head slows down
   auto decode = [&](long long u, int* b, int* hh, int* j) {
-    *hh = int(u % H); u /= H;
+    const bool vpass = u >= n_qk_units;
+    if (vpass) u -= n_qk_units;
+    const int H = vpass ? a.Hv : Hqk;
+    *hh = int(u % H) + (vpass ? Hqk : 0); u /= H;
     *b = int(u % a.B); u /= a.B;
     *j = int(u);
   };
@@ -95,8 +101,8 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     for (long long u = blockIdx.x; u < a.n_units; u += gridDim.x) {
       int b, hh, j;
       decode(u, &b, &hh, &j);
-      const CUtensorMap* tw = hh < a.Hq ? &tmWq : &tmWk;
-      const int wrow = (hh < a.Hq ? hh : hh - a.Hq) * kD;
+      const CUtensorMap* tw = hh < a.Hq ? &tmWq : (hh < a.Hq + a.Hkv ? &tmWk : &tmWv);
+      const int wrow = (hh < a.Hq ? hh : (hh < a.Hq + a.Hkv ? hh - a.Hq : hh - a.Hq - a.Hkv)) * kD;
       const int nt = n_tiles_of(j);
       for (int t = 0; t < nt; ++t) {
         const int tok0 = j * a.seg + t * kTileM;
@@ -145,8 +151,8 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     for (long long u = blockIdx.x; u < a.n_units; u += gridDim.x) {
       int b, hh, j;
       decode(u, &b, &hh, &j);
-      const bool is_q = hh < a.Hq;
-      const int h = is_q ? hh : hh - a.Hq;
+      const bool is_q = hh < a.Hq, is_v = hh >= a.Hq + a.Hkv;
+      const int h = is_q ? hh : (is_v ? hh - a.Hq - a.Hkv : hh - a.Hq);
       const int nt = n_tiles_of(j);
       float seg_max = -CUDART_INF_F, seg_min = CUDART_INF_F;       // channel `tid` over the segment (query heads)
       for (int t = 0; t < nt; ++t, ++tile_no) {
@@ -161,7 +167,7 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         tc_fence_before();
         mbar_arrive(&bars->acc_empty[as]);                         // the accumulator is in registers: its stage is free
         float* x = reinterpret_cast<float*>(acc);
-        if (a.cosT != nullptr && tok < a.n) {
+        if (a.cosT != nullptr && !is_v && tok < a.n) {
           // rotary embedding, rotate-half form: channel i pairs with channel i + 64
           const float4* c4 = reinterpret_cast<const float4*>(a.cosT + size_t(tok) * 64);
           const float4* s4 = reinterpret_cast<const float4*>(a.sinT + size_t(tok) * 64);
@@ -182,11 +188,13 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 #pragma unroll
         for (int i = 0; i < 64; ++i) w[i] = pack2<kF16>(x[2 * i], x[2 * i + 1]);
         if (tok < a.n) {
-          uint16_t* orow = is_q ? a.Q + b * a.qsb + h * a.qsh + int64_t(tok) * a.qst : a.K + b * a.ksb + h * a.ksh + int64_t(tok) * a.kst;
+          uint16_t* orow = is_q ? a.Q + b * a.qsb + h * a.qsh + int64_t(tok) * a.qst
+                         : (is_v ? a.V + b * a.vsb + h * a.vsh + int64_t(tok) * a.vst : a.K + b * a.ksb + h * a.ksh + int64_t(tok) * a.kst);
           uint4* dst = reinterpret_cast<uint4*>(orow);
 #pragma unroll
           for (int i = 0; i < 16; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
         }
+        if (is_v) continue;                                        // values: Eq. 1 alone, Algorithm 1 takes nothing from them
         // the rounded row goes to shared memory; then every thread scans one channel over the tile's rows
         uint32_t* trow = reinterpret_cast<uint32_t*>(tileT + row * kTStride);
 #pragma unroll
@@ -253,15 +261,17 @@ bool make_map3(CUtensorMap* map, const void* base, int d_model, long long rows, 
 
 }  // namespace
 
-int launch_project(const cp_params& p, const Dims& m, const void* X, const void* Wq, const void* Wk, const float* cosT,
-                   const float* sinT, int d_model, void* Q, void* K, char* ws, cudaStream_t st) {
+int launch_project(const cp_params& p, const Dims& m, const void* X, const void* Wq, const void* Wk, const void* Wv,
+                   const float* cosT, const float* sinT, int d_model, void* Q, void* K, void* V, char* ws, cudaStream_t st) {
   const bool f16 = p.dtype == CP_F16;
   if (!((p.dtype == CP_BF16 || f16) && m.d == kD && m.seg % kTileM == 0 && (m.blk == 32 || m.blk == 64 || m.blk == 128) &&
         d_model % kKB == 0 && d_model >= kKB && m.n >= kTileM))
     return CP_ERR_UNSUPPORTED;
   const WsLayout w = ws_layout(m);
   ProjArgs a;
-  a.Q = static_cast<uint16_t*>(Q); a.K = static_cast<uint16_t*>(K);
+  a.Q = static_cast<uint16_t*>(Q); a.K = static_cast<uint16_t*>(K); a.V = static_cast<uint16_t*>(V);
+  a.vsb = p.v_stride[0]; a.vsh = p.v_stride[1]; a.vst = p.v_stride[2];
+  a.Hv = (Wv != nullptr) ? m.Hkv : 0;
   a.qsb = p.q_stride[0]; a.qsh = p.q_stride[1]; a.qst = p.q_stride[2];
   a.ksb = p.k_stride[0]; a.ksh = p.k_stride[1]; a.kst = p.k_stride[2];
   a.cosT = cosT; a.sinT = sinT;
@@ -270,11 +280,13 @@ int launch_project(const cp_params& p, const Dims& m, const void* X, const void*
   a.kabs = reinterpret_cast<float*>(ws + w.kabs);
   a.st = reinterpret_cast<DeviceStatus*>(ws);
   a.B = m.B; a.Hq = m.Hq; a.Hkv = m.Hkv; a.n = m.n; a.seg = m.seg; a.blk = m.blk; a.n1 = m.n1; a.n2 = m.n2; a.d_model = d_model;
-  a.n_units = (long long)m.B * (m.Hq + m.Hkv) * m.n1;
-  CUtensorMap tmX, tmWq, tmWk;
+  a.n_units = (long long)m.B * (m.Hq + m.Hkv + a.Hv) * m.n1;
+  CUtensorMap tmX, tmWq, tmWk, tmWv;
   if (!make_map3(&tmX, X, d_model, m.n, m.B, f16) || !make_map3(&tmWq, Wq, d_model, (long long)m.Hq * kD, 1, f16) ||
       !make_map3(&tmWk, Wk, d_model, (long long)m.Hkv * kD, 1, f16))
     return CP_ERR_CUDA;
+  if (Wv == nullptr) tmWv = tmWk;
+  else if (!make_map3(&tmWv, Wv, d_model, (long long)m.Hkv * kD, 1, f16)) return CP_ERR_CUDA;
   auto kern = f16 ? project_sm100_kernel<true> : project_sm100_kernel<false>;
   const int smem = kSmemBar + int(sizeof(ProjBars)) + 1024;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CP_ERR_CUDA;
@@ -282,7 +294,7 @@ int launch_project(const cp_params& p, const Dims& m, const void* X, const void*
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return CP_ERR_CUDA;
   const unsigned grid = unsigned(a.n_units < sms ? a.n_units : sms);
-  kern<<<grid, kThreads, smem, st>>>(tmX, tmWq, tmWk, a);
+  kern<<<grid, kThreads, smem, st>>>(tmX, tmWq, tmWk, tmWv, a);
   return check_launch();
 }
 

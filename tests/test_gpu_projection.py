@@ -77,3 +77,29 @@ def test_projection_rejects_shapes_outside_its_envelope():
     with pytest.raises(cp.CritiPrefillError) as e:
         cp.project_qk(prob, X, W, W[:128].contiguous(), ws)
     assert e.value.status == 3
+
+
+@pytest.mark.parametrize("B,n,d_model,Hq,Hkv,seg,blk,dtype", [
+    (1, 1024, 256, 4, 2, 256, 64, "bf16"),
+    (2, 1000, 192, 2, 1, 128, 32, "f16"),                # batch 2, ragged length
+])
+def test_value_projection_in_the_same_launch(B, n, d_model, Hq, Hkv, seg, blk, dtype):
+    d = 128
+    X, Wq, Wk = _inputs(B, n, d_model, Hq, Hkv, d, dtype, seed=7)
+    _, _, Wv = _inputs(B, n, d_model, Hq, Hkv, d, dtype, seed=8)
+    cos, sin = oracle.rope_tables(n, d)
+    prob = cp.Problem(B, Hq, Hkv, n, d, seg, blk, max(seg // blk, 8), dtype=X.dtype)
+    ws, ws2 = cp.alloc_workspace(prob), cp.alloc_workspace(prob)
+    cd, sd = torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda()
+    Q, K, V = cp.project_qkv(prob, X.cuda(), Wq.cuda(), Wk.cuda(), Wv.cuda(), ws, rope_cos=cd, rope_sin=sd)
+    assert cp.device_status(ws) == 0
+    # V = W_V X (Eq. 1), unrotated: fp64 reference on the same bits, one rounding + fp32 accumulation
+    V_ref = oracle.project_v(X, Wv, d)
+    ulp = 2.0 ** -8 if dtype == "bf16" else 2.0 ** -11
+    err = np.abs(V.float().cpu().numpy().astype(np.float64) - V_ref)
+    assert (err <= ulp * np.abs(V_ref) + 2e-5 * np.sqrt(d_model)).all(), err.max()
+    # Q, K and the representatives are what the two-matrix call produces, bit for bit
+    Q2, K2 = cp.project_qk(prob, X.cuda(), Wq.cuda(), Wk.cuda(), ws2, rope_cos=cd, rope_sin=sd)
+    assert torch.equal(Q, Q2) and torch.equal(K, K2)
+    torch.cuda.synchronize()
+    assert torch.equal(ws[256:], ws2[256:])
