@@ -1,14 +1,15 @@
-// Upstream fusion: the query / key projections of Eq. 1 (Q = W_Q X, K = W_K X) with rotary position embedding, whose
+// Upstream fusion: the projections of Eq. 1 (Q = W_Q X, K = W_K X, optionally V = W_V X) with rotary position embedding on Q and K, whose
 // epilogue also produces the representatives of Algorithm 1, lines 3-8 (per-channel max / min of every query segment and
 // key block), so that critiprefill_estimate can skip its own pass over Q and K.
 //
-// GEMM on the tcgen05 tensor cores: D[128 tokens x 128 channels] = X_tile[128 x d_model] * W_head[128 x d_model]^T, one
-// output tile = 128 tokens of one head.  A work unit is (batch, head, segment): its seg/128 token tiles run back to
-// back on one CTA, so the segment's running max / min stay on chip.  Warps 0-3: epilogue (one thread per token row:
-// tensor-memory load, rotation, rounding, stores; then one thread per channel for the column scans), warp 4: TMA
-// producer (X and W tiles of 64 d_model columns, 5-stage ring, 128-byte swizzle), warp 5: MMA issuer; 4 accumulator
-// stages of 128 columns in tensor memory let the epilogue of one tile run under the main loop of the next.
-// Every wait is bounded.
+// GEMM on the tcgen05 tensor cores: D[128 tokens x 128 channels] = X_tile[128 x d_model] * W_head[128 x d_model]^T per
+// head; an output tile is 128 tokens of two adjacent heads of one kind (one head where a kind has an odd head count),
+// so that both heads share the X operand of every MMA.  A work unit is (batch, head group, segment): its seg/128 token
+// tiles run back to back on one CTA, so the segment's running max / min stay on chip.  Warps 0-3: epilogue (one thread
+// per token row: tensor-memory load, rotation, rounding, stores; then one thread per channel for the column scans), warp 4:
+// TMA producer (X and W tiles of 64 d_model columns, 128-byte swizzle), warp 5: MMA issuer; the accumulator stages in
+// tensor memory let the epilogue of one tile run under the main loop of the next.  The value heads (Eq. 1, no rotation, no
+// representatives) follow the query / key units as a pass of their own.  Every wait is bounded.
 #include "sm100_ptx.cuh"
 
 namespace cp {
@@ -19,15 +20,21 @@ constexpr int kD = 128;                       // head_dim = channels per output 
 constexpr int kTileM = 128;                   // tokens per output tile
 constexpr int kKB = 64;                       // d_model columns per pipeline stage (one 128-byte swizzled row)
 constexpr int kOpBytes = 128 * kKB * 2;       // one operand tile of a stage: 128 rows x 64 columns, 16-bit
-constexpr int kStageBytes = 2 * kOpBytes;     // X tile + W tile
-constexpr int kRing = 5;
-constexpr int kAcc = 4;                       // accumulator stages (4 x 128 columns)
 constexpr int kTStride = 132;                 // row stride (16-bit elements) of the transposition tile: conflict-free column reads
-constexpr int kSmemT = kRing * kStageBytes;
-constexpr int kSmemBar = kSmemT + kTileM * kTStride * 2;
+constexpr int kMaxRing = 5, kMaxAcc = 4;
+// kNH = heads per output tile.  Two adjacent heads of one kind share the X operand of every MMA (M128 N256 K16): a stage
+// then carries 16 KB of X for 32 KB of W instead of 16 + 16, which takes a quarter off the shared-memory and L2 traffic per
+// FLOP; the ring has 4 stages of 48 KB instead of 5 of 32 KB and tensor memory holds 2 accumulator stages of 256 columns.
+template <int kNH> struct Geo {
+  static constexpr int kStageBytes = (1 + kNH) * kOpBytes;     // X tile + W tile(s)
+  static constexpr int kRing = kNH == 2 ? 4 : 5;
+  static constexpr int kAcc = 4 / kNH;                         // accumulator stages (512 columns in all)
+  static constexpr int kSmemT = kRing * kStageBytes;
+  static constexpr int kSmemBar = kSmemT + kTileM * kTStride * 2;
+};
 
 struct ProjBars {
-  unsigned long long full[kRing], empty[kRing], acc_full[kAcc], acc_empty[kAcc];
+  unsigned long long full[kMaxRing], empty[kMaxRing], acc_full[kMaxAcc], acc_empty[kMaxAcc];
   uint32_t tmem_base;
   volatile int abort_flag;
   float red[4];
@@ -52,7 +59,7 @@ template <bool kF16> __device__ __forceinline__ float elem_to_f32(uint16_t v) {
 
 __device__ __forceinline__ void bar_sync_epilogue() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-template <bool kF16>
+template <bool kF16, int kNH>
 __global__ void __launch_bounds__(kThreads, 1)
 project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmWq,
                      const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmWv, const ProjArgs a) {
@@ -60,8 +67,9 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t smem_base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (smem_base - raw);
-  uint16_t* tileT = reinterpret_cast<uint16_t*>(sm + kSmemT);
-  ProjBars* bars = reinterpret_cast<ProjBars*>(sm + kSmemBar);
+  constexpr int kStageBytes = Geo<kNH>::kStageBytes, kRing = Geo<kNH>::kRing, kAcc = Geo<kNH>::kAcc;
+  uint16_t* tileT = reinterpret_cast<uint16_t*>(sm + Geo<kNH>::kSmemT);
+  ProjBars* bars = reinterpret_cast<ProjBars*>(sm + Geo<kNH>::kSmemBar);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
@@ -78,7 +86,7 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   tc_fence_after();
   const uint32_t tm = bars->tmem_base;
 
-  const int Hqk = a.Hq + a.Hkv;            // heads in the order query, key, value
+  const int Hqk = (a.Hq + a.Hkv) / kNH;    // head groups (kNH adjacent heads of one kind) in the order query, key, value
   const long long n_qk_units = (long long)a.B * Hqk * a.n1;
   const int tiles_per_seg = a.seg / kTileM;
   const int n_kb = a.d_model / kKB;
@@ -88,8 +96,8 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
   auto decode = [&](long long u, int* b, int* hh, int* j) {
     const bool vpass = u >= n_qk_units;
     if (vpass) u -= n_qk_units;
-    const int H = vpass ? a.Hv : Hqk;
-    *hh = int(u % H) + (vpass ? Hqk : 0); u /= H;
+    const int H = vpass ? a.Hv / kNH : Hqk;
+    *hh = (int(u % H) + (vpass ? Hqk : 0)) * kNH; u /= H;      // first head of the group
     *b = int(u % a.B); u /= a.B;
     *j = int(u);
   };
@@ -113,7 +121,7 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
             const uint32_t dst = smem_base + s * kStageBytes;
             mbar_expect_tx(&bars->full[s], kStageBytes);
             tma_load_3d(dst, &tmX, &bars->full[s], kb * kKB, tok0, b);            // rows past n arrive as zeros
-            tma_load_3d(dst + kOpBytes, tw, &bars->full[s], kb * kKB, wrow, 0);
+            tma_load_3d(dst + kOpBytes, tw, &bars->full[s], kb * kKB, wrow, 0);   // 128 * kNH weight rows
           }
           __syncwarp();
         }
@@ -123,6 +131,8 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
     // ---------------- MMA issuer
     uint32_t it = 0, tile_no = 0;
     const uint64_t base = desc_base(16);
+    // M = 128, N = 128 * kNH (bits 17-22 hold N / 8)
+    constexpr uint32_t kIdesc = (Idesc<kF16>::qk & ~(0x3fu << 17)) | ((uint32_t(kD * kNH) >> 3) << 17);
     for (long long u = blockIdx.x; u < a.n_units; u += gridDim.x) {
       int b, hh, j;
       decode(u, &b, &hh, &j);
@@ -137,7 +147,7 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
           const uint32_t xa = smem_base + s * kStageBytes, wa = xa + kOpBytes;
 #pragma unroll
           for (int kk = 0; kk < kKB / 16; ++kk)
-            umma_ss(tm + as * kD, desc_at(base, xa + kk * 32), desc_at(base, wa + kk * 32), Idesc<kF16>::qk, (kb > 0 || kk > 0) ? 1u : 0u);
+            umma_ss(tm + as * kD * kNH, desc_at(base, xa + kk * 32), desc_at(base, wa + kk * 32), kIdesc, (kb > 0 || kk > 0) ? 1u : 0u);
           umma_commit(&bars->empty[s]);
         }
         umma_commit(&bars->acc_full[as]);
@@ -152,20 +162,27 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
       int b, hh, j;
       decode(u, &b, &hh, &j);
       const bool is_q = hh < a.Hq, is_v = hh >= a.Hq + a.Hkv;
-      const int h = is_q ? hh : (is_v ? hh - a.Hq - a.Hkv : hh - a.Hq);
+      const int h0 = is_q ? hh : (is_v ? hh - a.Hq - a.Hkv : hh - a.Hq);   // first head of the group within its kind
       const int nt = n_tiles_of(j);
-      float seg_max = -CUDART_INF_F, seg_min = CUDART_INF_F;       // channel `tid` over the segment (query heads)
+      float seg_max[kNH], seg_min[kNH];                            // channel `tid` over the segment (query heads)
+#pragma unroll
+      for (int sub = 0; sub < kNH; ++sub) { seg_max[sub] = -CUDART_INF_F; seg_min[sub] = CUDART_INF_F; }
       for (int t = 0; t < nt; ++t, ++tile_no) {
         const uint32_t as = tile_no % kAcc;
         const int tok0 = j * a.seg + t * kTileM;
         const int tok = tok0 + row;
         if (!mbar_wait(&bars->acc_full[as], (tile_no / kAcc) & 1, &bars->abort_flag, a.st, 73)) return;
         tc_fence_after();
+#pragma unroll
+       for (int sub = 0; sub < kNH; ++sub) {                       // the heads of the group, 128 accumulator columns each
+        const int h = h0 + sub;
         uint32_t acc[128];
-        tmem_ld128(t_row + as * kD, acc);
+        tmem_ld128(t_row + as * kD * kNH + sub * kD, acc);
         tmem_wait_ld();
-        tc_fence_before();
-        mbar_arrive(&bars->acc_empty[as]);                         // the accumulator is in registers: its stage is free
+        if (sub == kNH - 1) {
+          tc_fence_before();
+          mbar_arrive(&bars->acc_empty[as]);                       // the accumulator is in registers: its stage is free
+        }
         float* x = reinterpret_cast<float*>(acc);
         if (a.cosT != nullptr && !is_v && tok < a.n) {
           // rotary embedding, rotate-half form: channel i pairs with channel i + 64
@@ -205,7 +222,7 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
         if (is_q) {
           for (int r = 0; r < rows_valid; ++r) {
             const float v = elem_to_f32<kF16>(tileT[r * kTStride + c]);
-            seg_max = fmaxf(seg_max, v); seg_min = fminf(seg_min, v);
+            seg_max[sub] = fmaxf(seg_max[sub], v); seg_min[sub] = fminf(seg_min[sub], v);
           }
         } else {
           // key heads: one (max, min) per block of blk tokens, written straight away; kabs = largest magnitude of the block's summaries
@@ -230,11 +247,15 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
           }
         }
         bar_sync_epilogue();                                       // the tile may be overwritten by the next one
+       }
       }
       if (is_q) {
-        const long long unit = ((long long)b * a.Hq + h) * a.n1 + j;
-        a.Qmax[unit * kD + tid] = uint16_t(pack2<kF16>(seg_max, 0.f) & 0xffffu);
-        a.Qmin[unit * kD + tid] = uint16_t(pack2<kF16>(seg_min, 0.f) & 0xffffu);
+#pragma unroll
+        for (int sub = 0; sub < kNH; ++sub) {
+          const long long unit = ((long long)b * a.Hq + h0 + sub) * a.n1 + j;
+          a.Qmax[unit * kD + tid] = uint16_t(pack2<kF16>(seg_max[sub], 0.f) & 0xffffu);
+          a.Qmin[unit * kD + tid] = uint16_t(pack2<kF16>(seg_min[sub], 0.f) & 0xffffu);
+        }
       }
     }
   }
@@ -247,12 +268,12 @@ project_sm100_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_const
 }
 
 // rows x d_model 16-bit matrix, row-major; box = 64 columns x 128 rows; third dimension = batches of `rows` rows
-bool make_map3(CUtensorMap* map, const void* base, int d_model, long long rows, long long batches, bool f16) {
+bool make_map3(CUtensorMap* map, const void* base, int d_model, long long rows, long long batches, bool f16, int box_rows = 128) {
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[3] = {cuuint64_t(d_model), cuuint64_t(rows), cuuint64_t(batches)};
   cuuint64_t strides[2] = {cuuint64_t(d_model) * 2, cuuint64_t(rows) * cuuint64_t(d_model) * 2};
-  cuuint32_t box[3] = {cuuint32_t(kKB), cuuint32_t(rows < 128 ? rows : 128), 1};
+  cuuint32_t box[3] = {cuuint32_t(kKB), cuuint32_t(rows < box_rows ? rows : box_rows), 1};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
             box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -280,15 +301,18 @@ int launch_project(const cp_params& p, const Dims& m, const void* X, const void*
   a.kabs = reinterpret_cast<float*>(ws + w.kabs);
   a.st = reinterpret_cast<DeviceStatus*>(ws);
   a.B = m.B; a.Hq = m.Hq; a.Hkv = m.Hkv; a.n = m.n; a.seg = m.seg; a.blk = m.blk; a.n1 = m.n1; a.n2 = m.n2; a.d_model = d_model;
-  a.n_units = (long long)m.B * (m.Hq + m.Hkv + a.Hv) * m.n1;
+  // two heads per output tile where every kind has an even head count (see Geo)
+  const int nh = (m.Hq % 2 == 0 && m.Hkv % 2 == 0) ? 2 : 1;
+  a.n_units = (long long)m.B * ((m.Hq + m.Hkv + a.Hv) / nh) * m.n1;
   CUtensorMap tmX, tmWq, tmWk, tmWv;
-  if (!make_map3(&tmX, X, d_model, m.n, m.B, f16) || !make_map3(&tmWq, Wq, d_model, (long long)m.Hq * kD, 1, f16) ||
-      !make_map3(&tmWk, Wk, d_model, (long long)m.Hkv * kD, 1, f16))
+  if (!make_map3(&tmX, X, d_model, m.n, m.B, f16) || !make_map3(&tmWq, Wq, d_model, (long long)m.Hq * kD, 1, f16, 128 * nh) ||
+      !make_map3(&tmWk, Wk, d_model, (long long)m.Hkv * kD, 1, f16, 128 * nh))
     return CP_ERR_CUDA;
   if (Wv == nullptr) tmWv = tmWk;
-  else if (!make_map3(&tmWv, Wv, d_model, (long long)m.Hkv * kD, 1, f16)) return CP_ERR_CUDA;
-  auto kern = f16 ? project_sm100_kernel<true> : project_sm100_kernel<false>;
-  const int smem = kSmemBar + int(sizeof(ProjBars)) + 1024;
+  else if (!make_map3(&tmWv, Wv, d_model, (long long)m.Hkv * kD, 1, f16, 128 * nh)) return CP_ERR_CUDA;
+  auto kern = nh == 2 ? (f16 ? project_sm100_kernel<true, 2> : project_sm100_kernel<false, 2>)
+                      : (f16 ? project_sm100_kernel<true, 1> : project_sm100_kernel<false, 1>);
+  const int smem = (nh == 2 ? Geo<2>::kSmemBar : Geo<1>::kSmemBar) + int(sizeof(ProjBars)) + 1024;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return CP_ERR_CUDA;
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
