@@ -88,6 +88,7 @@ struct Args {
   int dense;
   int n_units;
   int o_vec32;                  // O rows are 32-byte aligned: the epilogue may use 32-byte stores
+  int emul;                     // long units: part of the exponentials on the FMA pipes (see launch_attention_sm100)
   int withhold_v;               // test hook: the producer never issues V tiles, so a bounded wait must expire
   unsigned int* work_counter;   // next unit to hand out (zeroed by the host before the launch)
 };
@@ -363,8 +364,8 @@ __device__ __forceinline__ void softmax_role(const Args& a, Bars* bars, int whic
       const float2 c2 = make_float2(c, c), nm2 = make_float2(neg_mc, neg_mc);
       float2 sum2 = make_float2(0.f, 0.f);
       uint32_t pk[64];
-      if (kind == kMaskNone) {
-        // unmasked tile: every kEmulEvery-th pair takes the polynomial path, the rest the MUFU
+      if (kind == kMaskNone && a.emul) {
+        // unmasked tile of a long unit: every kEmulEvery-th pair takes the polynomial path, the rest the MUFU
 #pragma unroll
         for (int i = 0; i < 128; i += 2) {
           const float2 xx = __ffma2_rn(make_float2(s[i], s[i + 1]), c2, nm2);
@@ -687,6 +688,10 @@ int launch_attention_sm100(const cp_params& p, const Dims& m, const void* Q, con
     return CP_ERR_CUDA;
   a.n_units = int(units);
   a.withhold_v = (p.flags & CP_FLAG_TEST_WITHHOLD_V) ? 1 : 0;
+  // Moving every kEmulEvery-th pair of exponentials from the MUFU to the FMA pipes pays where units are long and the
+  // kernel sits at the power cap (measured in 60-step loops: 1.6 % at 32 K/V tiles per unit) and costs where units are
+  // short (3 % at 8 tiles per unit, the paper's operating point); a unit streams at most k*blk/128 tiles.
+  a.emul = (dense || (long long)m.k * m.blk >= 12 * kTile) ? 1 : 0;
   a.o_vec32 = (reinterpret_cast<uintptr_t>(O) % 32 == 0 && p.o_stride[0] % 16 == 0 && p.o_stride[1] % 16 == 0 && p.o_stride[2] % 16 == 0) ? 1 : 0;
   a.work_counter = reinterpret_cast<unsigned int*>(reinterpret_cast<char*>(st) + 128);   // inside the status block
   if (cudaMemsetAsync(a.work_counter, 0, sizeof(unsigned int), s) != cudaSuccess) return CP_ERR_CUDA;
