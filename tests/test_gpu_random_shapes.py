@@ -64,3 +64,63 @@ def test_random_shape_matches_oracle(seed):
     # 16-bit outputs: the stated absolute bound on unit-scale values, relative beyond |O| = 2 (output spacing)
     tol = {"f32": 1e-5, "f16": 2e-3, "bf16": 1e-2}[dtype]
     assert (err / np.maximum(1.0, np.abs(O_ref) / 2)).max() <= tol, (c, float(err.max()))
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_valid_lists_and_dense(seed):
+    """critiprefill_attention on lists it did not get from critiprefill_select (Algorithm 2 takes any index set): empty
+    lists, any visible blocks, a lone diagonal block, the usual form with fewer past blocks, every other diagonal block --
+    drawn per (head, segment); and critiprefill_dense_attention on the same inputs."""
+    rng = np.random.default_rng(10_000 + seed)
+    dtype = str(rng.choice(["bf16", "bf16", "f16", "f32"]))
+    d, blk = int(rng.choice([128, 128, 128, 64])), int(rng.choice([16, 32, 64, 128]))
+    r = min(int(rng.choice([1, 2, 4, 8])), 1024 // blk)
+    seg, n = blk * r, int(rng.integers(1, 2600))
+    Hkv, g, B = int(rng.choice([1, 2])), int(rng.choice([1, 2, 4])), int(rng.choice([1, 2]))
+    Hq, k = Hkv * g, r + int(rng.integers(0, 20))
+    flags = cp.FLAG_FORCE_SIMT if rng.integers(0, 6) == 0 else 0
+    n1, n2 = -(-n // seg), -(-n // blk)
+    idx = np.full((B, Hq, n1, k), -1, dtype=np.int32)
+    cnt = np.zeros((B, Hq, n1), dtype=np.int32)
+    for b in range(B):
+        for h in range(Hq):
+            for j in range(n1):
+                vis = min(n2, (j + 1) * r)
+                rj = vis - j * r
+                mode = int(rng.integers(0, 6))
+                if mode == 0:
+                    sel = []
+                elif mode == 1:
+                    sel = sorted(rng.choice(vis, size=min(k, vis, 1 + int(rng.integers(k))), replace=False).tolist())
+                elif mode == 2:
+                    sel = [j * r + int(rng.integers(rj))]
+                elif mode in (3, 4):
+                    m = min(k - rj, j * r)
+                    past = sorted(rng.choice(j * r, size=int(rng.integers(0, m + 1)), replace=False).tolist()) if j and m > 0 else []
+                    sel = past + list(range(j * r, vis))
+                else:
+                    sel = sorted(set(range(j * r, vis, 2)) | ({0} if j else set()))[:k]
+                cnt[b, h, j] = len(sel)
+                idx[b, h, j, :len(sel)] = sel
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[dtype]
+    Q, K, V = make_uniform_qkv(B, Hq, Hkv, n, d, dtype=dtype, seed=seed)
+    prob = cp.Problem(B, Hq, Hkv, n, d, seg, blk, k, tdt, flags=flags)
+    ws = cp.alloc_workspace(prob)
+    Qd, Kd, Vd = Q.cuda(), K.cuda(), V.cuda()
+    O, lse = cp.attention(prob, Qd, Kd, Vd, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), ws, want_lse=True)
+    assert cp.device_status(ws) == 0
+    sm = f32(1.0 / np.sqrt(d))
+    tol = {"f32": 1e-5, "f16": 2e-3, "bf16": 1e-2}[dtype]
+    O_ref, lse_ref = oracle.sparse_attention(Q, K, V, idx, cnt, seg, blk, sm)
+    err = np.abs(O.float().cpu().numpy().astype(np.float64) - O_ref)
+    assert (err / np.maximum(1.0, np.abs(O_ref) / 2)).max() <= tol
+    none = np.isneginf(lse_ref)                                    # rows that see no key: zeros, lse = -inf
+    lg = lse.cpu().numpy()
+    assert np.array_equal(np.isneginf(lg), none) and (O.float().cpu().numpy()[none] == 0).all()
+    if (~none).any():
+        assert np.abs(lg[~none] - lse_ref[~none]).max() <= 2e-3
+    Od = cp.dense_attention(prob, Qd, Kd, Vd, ws)
+    assert cp.device_status(ws) == 0
+    Od_ref, _ = oracle.dense_attention(Q, K, V, sm)
+    errd = np.abs(Od.float().cpu().numpy().astype(np.float64) - Od_ref)
+    assert (errd / np.maximum(1.0, np.abs(Od_ref) / 2)).max() <= tol
