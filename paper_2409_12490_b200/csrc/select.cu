@@ -46,8 +46,10 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int lane, int warp, i
 // consecutive query heads' scores, and the one list is written for each of them.  n_sink / n_local: the first
 // n_sink blocks and the n_local blocks right before the segment get the largest possible key, so they are taken
 // before any scored block (the host has checked that they fit into the k - r free slots).
+// Resident CTAs per SM are set by registers: the kernel waits on barriers most of the time, so 16 keys per thread are held to 64
+// registers (4 CTAs instead of the 3 that 80 registers allow: 13 % faster at n2 = 4096; 48 registers spill and are slower).
 template <int KPT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, KPT <= 4 ? 5 : (KPT <= 16 ? 4 : 2))
 select_kernel(const double* __restrict__ S, int32_t* __restrict__ idx, int32_t* __restrict__ cnt,
               int n1, int n2, int r, int k, int pool, int n_sink, int n_local, int past_fixed) {
   __shared__ unsigned int hist[256];
