@@ -54,6 +54,7 @@ struct LseBars {
   unsigned long long kv_full[kSlots], kv_empty[kSlots], acc_full[kStages], acc_empty[kStages];
   uint32_t tmem_base;
   volatile int abort_flag;
+  int next_list;                 // exact pass: the lists are handed out to the warps as they become free
   float kabs_red[kWarps];
 };
 
@@ -131,6 +132,7 @@ lse_sm100_kernel(const __grid_constant__ CUtensorMap tmKmax, const __grid_consta
     for (int i = 0; i < kSlots; ++i) { mbar_init(&bars->kv_full[i], 1); mbar_init(&bars->kv_empty[i], 1); }
     for (int i = 0; i < kStages; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 128); }
     bars->abort_flag = 0;
+    bars->next_list = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 8 && lane == 0) { prefetch_tmap(&tmKmax); prefetch_tmap(&tmKmin); }
@@ -306,7 +308,14 @@ lse_sm100_kernel(const __grid_constant__ CUtensorMap tmKmax, const __grid_consta
     uint16_t* queue = queues + warp * kQueue;
     double* qs = reinterpret_cast<double*>(sm + kSmemKV) + warp * 8 * kQS;   // this warp's B operand, in the idle K ring
     const double es_d = double(a.es);
-    for (int l = warp; l < kLists; l += kWarps) {
+    for (;;) {
+      // lists differ a lot in length (a few rows near their maximum flag most of the blocks), so they are taken first
+      // come, first served (a fixed round-robin left the slowest warp 25 % behind; halving the lists for a finer grain
+      // costs more in B-operand set-up than it balances)
+      int l = 0;
+      if (lane == 0) l = atomicAdd(&bars->next_list, 1);
+      l = __shfl_sync(0xffffffffu, l, 0);
+      if (l >= kLists) break;
       const int cg = l >> 1, kr = l & 1;
       if (row_seg(cg * 8) >= a.n1) continue;              // the group's first segment does not exist: nothing flagged
       // B operand: the 8 rows of the group widened to fp64, [row][k-step][lane-in-quad][4 channels]
