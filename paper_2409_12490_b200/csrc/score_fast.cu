@@ -10,7 +10,7 @@
 namespace cp {
 namespace {
 
-constexpr int kThreads = 256;   // 8 warps x <= 128 registers: two CTAs per SM, so one CTA's set-up and tile epilogues run under the other's MMAs
+constexpr int kThreads = 256;   // 8 warps x <= 85 registers: three CTAs per SM, so a CTA's set-up and tile epilogues run under the others' MMAs
 constexpr int kWarps = kThreads / 32;
 #ifndef CP_SCORE_FAST_MIN
 #define CP_SCORE_FAST_MIN 3000000
@@ -25,7 +25,7 @@ constexpr int kG = 4;                       // segments per CTA: one MMA column 
 // all four logits l1..l4 in its accumulators (Kmax product: cx, Kmin product: cn; even element: Qmax, odd:
 // Qmin) and finishes the element without shared memory.
 template <typename T, int D, int U>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 3)
 score_visible_kernel(const T* __restrict__ Qmax, const T* __restrict__ Qmin, const T* __restrict__ Kmax,
                      const T* __restrict__ Kmin, const double* __restrict__ stats, const double* __restrict__ S_prev,
                      double* __restrict__ S_out, int Hq, int g, int n1, int n2, int seg, int blk, double est_scale,
@@ -183,8 +183,9 @@ int launch_visible(const Dims& m, const char* ws, const WsLayout& w, const doubl
 template <typename T>
 int launch_visible_t(const Dims& m, const char* ws, const WsLayout& w, const double* S_prev, double* S_out,
                      double est_scale, double alpha, int fuse, cudaStream_t st) {
-  // (four heads per CTA need 154 registers and leave room for one CTA of 12 warps per SM: measured 3 % slower at n2 = 4096)
-  if (m.g % 2 == 0) return launch_visible<T, 2>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, st);
+  // One head per CTA: 80 registers, three CTAs of 8 warps per SM.  More heads per CTA amortise the widening of the A operand
+  // over more MMAs but leave fewer CTAs to overlap (measured at n2 = 4096: U = 4 with one CTA of 12 warps 0.69 ms, U = 2 with two
+  // CTAs 0.65 ms, U = 1 with three 0.62 ms; four CTAs at 64 registers spill and gain nothing).
   return launch_visible<T, 1>(m, ws, w, S_prev, S_out, est_scale, alpha, fuse, st);
 }
 
